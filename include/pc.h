@@ -1,0 +1,161 @@
+/*
+ * libpc: the attention hot path of ParallelComp (arXiv 2502.14317, Sec. 3.1) for one
+ * layer on one B200 (sm_100a).  C ABI, plain pointers and sizes.
+ *
+ * Notation.  A long input is cut into C chunks; every chunk is followed by the same
+ * query window of w tokens, so a chunk holds L = ctx + w tokens, with RoPE positions
+ * 0..L-1 restarting in every chunk (position reuse).  Hq query heads, Hkv key/value
+ * heads, G = Hq / Hkv, head size d.  m chunks and k tokens per (kept chunk, kv-head)
+ * survive eviction; the compressed cache has Nk = m * k entries per kv-head.
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers, 16-byte aligned, bf16 unless stated
+ *     otherwise; d is the contiguous dimension; strides are in elements and must be
+ *     multiples of 8.  Descriptor structs and stride arrays are HOST memory.
+ *   - The caller owns every buffer.  The library allocates no device memory and keeps
+ *     no state between calls; scratch comes from the caller's workspace, sized by the
+ *     matching *_workspace_bytes query (host function, no GPU work).
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream) and return without synchronising.  Index outputs of one call
+ *     are device inputs of the next, so the five calls chain on one stream with no
+ *     host round trip.
+ *   - Return value: PC_OK or a negative pc_status.  Argument errors are found on the
+ *     host before anything is launched; nothing is written in that case.
+ *   - `status_word` (device int32, may be NULL) is left untouched on success; a kernel
+ *     whose bounded wait on a copy or tensor-core barrier ran out stores a non-zero
+ *     code there and the results of that call are undefined.  The caller clears it and
+ *     reads it after synchronising.  No kernel spins without a limit.
+ *   - Supported: d in {64, 128}; Hq % Hkv == 0; w % 8 == 0; 8 <= w <= 128; w < L;
+ *     G * w <= 256 rows are handled per pass (larger groups take several passes).
+ */
+#ifndef PC_H_
+#define PC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define PC_API __attribute__((visibility("default")))
+#else
+#define PC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PC_OK = 0,
+  PC_ERR_INVALID_ARG = -1,   /* null pointer, bad size, misaligned pointer or stride      */
+  PC_ERR_UNSUPPORTED = -2,   /* shape outside the supported set, or device is not sm_100  */
+  PC_ERR_WORKSPACE = -3,     /* workspace missing or smaller than *_workspace_bytes       */
+  PC_ERR_CUDA = -4,          /* a CUDA runtime / driver call failed                       */
+  PC_ERR_TIMEOUT = -5        /* value stored in status_word by a kernel whose wait ran out */
+} pc_status;
+
+/* Text for a status code (static storage). */
+PC_API const char* pc_status_string(int32_t status);
+
+/* Library version, major * 1000 + minor. */
+PC_API int32_t pc_version(void);
+
+/* ------------------------------------------------------------------------------------
+ * Chunk-local causal attention with position reuse and fused query-window scores.
+ * Paper: Sec. 3.1 "Parallel attention" (chunking, Eq. 1-2) and "Parallel KV cache
+ * eviction" (Eq. 5-6).
+ *
+ * For every chunk c and q-head h (kv-head h / G), with q', k' = RoPE(q), RoPE(k) at the
+ * token's chunk-local position (pairs (t, t + d/2), angle p * theta^(-2t/d)) rounded to
+ * bf16:
+ *     A = softmax(q' k'^T * scale + causal mask),  O = A v                      (Eq. 1-2)
+ *     win_score[c, hkv, j] = sum_{g < G} sum_{i = L-w}^{L-1} A[c, hkv*G+g, i, j]    (Eq. 6)
+ * The score is accumulated inside the attention kernel (second sweep of the window rows
+ * against the final log-sum-exp); it is not a separate launch.
+ *
+ * q [C,L,Hq,d], k, v [C,L,Hkv,d]: inputs before RoPE, addressed through the element
+ * strides (chunk, token, head) in the descriptor.
+ * o [C,L,Hq,d] (strides o_stride), k_rot [C,L,Hkv,d] contiguous (rotated keys, what the
+ * gather later copies; may be NULL, then it lives in the workspace), lse [C,Hq,L] fp32
+ * natural-log log-sum-exp of every row (may be NULL), win_score [C,Hkv,L] fp32,
+ * win_lse [C,Hq,w] fp32 (rows L-w..L-1).
+ */
+typedef struct {
+  int32_t C, L, w, Hq, Hkv, d;
+  float rope_theta;
+  float softmax_scale;                 /* 0 -> 1/sqrt(d) */
+  int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];   /* chunk, token, head; 0,0,0 -> contiguous */
+} pc_prefill_desc;
+
+PC_API size_t pc_chunk_prefill_attn_workspace_bytes(const pc_prefill_desc* desc, int32_t k_rot_in_workspace);
+
+PC_API int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const void* k, const void* v,
+                              void* o, void* k_rot, float* lse, float* win_score, float* win_lse,
+                              int32_t* status_word, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Stand-in for the chunk self-information I_c of Eq. 3 in a single-layer setting
+ * (the true I_c = -log P(X^q | X^c) needs the whole model; it enters pc_select_chunks
+ * as an input array).  chunk_score[c] = - mean over q-heads and window rows of
+ * win_lse[c, h, i].  Not part of the paper; used by the synthetic pipeline only.
+ * win_lse [C,Hq,w] fp32 -> chunk_score [C] fp32.
+ */
+PC_API int32_t pc_chunk_score_from_lse(const float* win_lse, int32_t C, int32_t Hq, int32_t w, float* chunk_score,
+                                void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Chunk eviction.  Paper: Sec. 3.1 "Chunk eviction", Eq. 3-4 (fixed-size queue keeping
+ * the chunks with the lowest self-information).
+ * Keeps the m best of C scores (lowest if lower_is_better != 0); ties go to the lower
+ * chunk id; NaN ranks worst; kept[m] lists the chunk ids in ascending order.
+ * 1 <= m <= C <= 1024.
+ */
+PC_API int32_t pc_select_chunks(const float* chunk_score, int32_t C, int32_t m, int32_t lower_is_better,
+                         int32_t* kept, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Token eviction per kept chunk and kv-head.  Paper: Sec. 3.1 "Parallel KV cache
+ * eviction", Eq. 7.
+ * For row (r, hkv), r < m: the k largest of win_score[kept[r], hkv, 0..n_cand) (window
+ * keys j >= n_cand are never candidates); ties go to the lower position; NaN ranks
+ * worst; -0 == +0.  idx[m,Hkv,k] int32 holds the positions in ascending order; if
+ * k > n_cand the tail is filled with -1.  `kept` is a device array (output of
+ * pc_select_chunks).  n_cand <= L, n_cand <= 32768.
+ */
+PC_API int32_t pc_select_tokens(const float* win_score, const int32_t* kept, int32_t C, int32_t m, int32_t Hkv,
+                         int32_t L, int32_t n_cand, int32_t k, int32_t* idx, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Compressed cache.  Paper: Eq. 7 (K[R], V[R]) and Eq. 9 (concatenation over chunks).
+ *     k_out[hkv, r*k + t, :] = k_src[kept[r], idx[r,hkv,t], hkv, :]     (same for v)
+ *     pos_out[hkv, r*k + t]  = idx[r,hkv,t]
+ * k_src (rotated keys) and v_src are [C,L,Hkv,d] addressed by kv_stride (chunk, token,
+ * head; host array; NULL -> contiguous); outputs are contiguous [Hkv, m*k, d] and
+ * [Hkv, m*k] int32 (pos_out may be NULL).  Entries with idx < 0 give zero rows and
+ * position -1.  Pure bit copy.
+ */
+PC_API int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t* kv_stride, int32_t L,
+                     const int32_t* kept, const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d,
+                     void* k_out, void* v_out, int32_t* pos_out, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Parallel (global) attention of the query window over the compressed multi-chunk
+ * cache.  Paper: Sec. 3.1 "Global attention", Eq. 9-11.
+ * For each of B sequences: the w window queries (rotated here at positions
+ * q_pos0..q_pos0+w-1, rounded to bf16) attend to all Nk cache entries of their kv-head
+ * (every kept key precedes the window, so no mask) and causally to the window's own w
+ * keys.  Keys arrive already rotated.  Split over key ranges with an fp32 merge.
+ * q_win [B,w,Hq,d]; k_cache, v_cache [B,Hkv,Nk,d]; k_win, v_win [B,w,Hkv,d];
+ * out [B,w,Hq,d] bf16; lse_out [B,Hq,w] fp32 natural log (may be NULL).  All contiguous.
+ */
+PC_API size_t pc_parallel_attn_workspace_bytes(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk);
+
+PC_API int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk,
+                         const void* q_win, int32_t q_pos0, float rope_theta, float softmax_scale,
+                         const void* k_cache, const void* v_cache, const void* k_win, const void* v_win,
+                         void* out, float* lse_out, int32_t* status_word, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PC_H_ */

@@ -1,0 +1,13 @@
+"""ParallelComp attention hot path for B200 (sm_100a): thin Python binding over libpc.so.
+
+The functions here only marshal arguments (torch tensors -> device pointers); every
+step of the path runs in the CUDA kernels behind the C ABI declared in include/pc.h.
+There is no CPU fallback: importing :mod:`paper_2502_14317_b200.binding` raises if the
+library is missing.
+"""
+from .binding import (  # noqa: F401
+    PcError, lib_path, load_library, version, status_string,
+    chunk_prefill_attn, chunk_prefill_attn_workspace_bytes, chunk_score_from_lse,
+    select_chunks, select_tokens, gather_kv, parallel_attn, parallel_attn_workspace_bytes,
+    hot_path,
+)

@@ -1,0 +1,264 @@
+"""ctypes binding for libpc.so.  Same names as the C entry points, minus the ``pc_`` prefix.
+
+Tensors are torch CUDA tensors; bf16 data is ``torch.bfloat16``.  Outputs and
+workspaces are allocated here with torch (device memory only) unless passed in.
+All calls enqueue on torch's current stream and do not synchronise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_float, c_int32, c_int64, c_size_t, c_void_p, c_char_p, POINTER, Structure
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+
+class PcError(RuntimeError):
+    pass
+
+
+class _PrefillDesc(Structure):
+    _fields_ = [("C", c_int32), ("L", c_int32), ("w", c_int32), ("Hq", c_int32), ("Hkv", c_int32), ("d", c_int32),
+                ("rope_theta", c_float), ("softmax_scale", c_float),
+                ("q_stride", c_int64 * 3), ("k_stride", c_int64 * 3), ("v_stride", c_int64 * 3),
+                ("o_stride", c_int64 * 3)]
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, "libpc.so")
+
+
+def load_library():
+    """Load libpc.so (built in-tree by ``python -m paper_2502_14317_b200.build``).  Fails loudly if absent."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = lib_path()
+    if not os.path.exists(path):
+        raise PcError(f"{path} not found: build it with `python -m paper_2502_14317_b200.build` "
+                      "(there is no fallback path)")
+    lib = ctypes.CDLL(path)
+    lib.pc_status_string.restype = c_char_p
+    lib.pc_status_string.argtypes = [c_int32]
+    lib.pc_version.restype = c_int32
+    lib.pc_chunk_prefill_attn_workspace_bytes.restype = c_size_t
+    lib.pc_chunk_prefill_attn_workspace_bytes.argtypes = [POINTER(_PrefillDesc), c_int32]
+    lib.pc_chunk_prefill_attn.restype = c_int32
+    lib.pc_chunk_prefill_attn.argtypes = [POINTER(_PrefillDesc)] + [c_void_p] * 10 + [c_size_t, c_void_p]
+    lib.pc_chunk_score_from_lse.restype = c_int32
+    lib.pc_chunk_score_from_lse.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
+    lib.pc_select_chunks.restype = c_int32
+    lib.pc_select_chunks.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
+    lib.pc_select_tokens.restype = c_int32
+    lib.pc_select_tokens.argtypes = [c_void_p, c_void_p] + [c_int32] * 6 + [c_void_p, c_void_p]
+    lib.pc_gather_kv.restype = c_int32
+    lib.pc_gather_kv.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_int32, c_void_p, c_void_p] + [c_int32] * 4 + \
+                                [c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.pc_parallel_attn_workspace_bytes.restype = c_size_t
+    lib.pc_parallel_attn_workspace_bytes.argtypes = [c_int32] * 6
+    lib.pc_parallel_attn.restype = c_int32
+    lib.pc_parallel_attn.argtypes = [c_int32] * 6 + [c_void_p, c_int32, c_float, c_float] + [c_void_p] * 8 + \
+                                    [c_size_t, c_void_p]
+    _LIB = lib
+    return lib
+
+
+def version() -> int:
+    return int(load_library().pc_version())
+
+
+def status_string(code: int) -> str:
+    return load_library().pc_status_string(int(code)).decode()
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise PcError(f"{what} failed: {status_string(rc)} ({rc})")
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream():
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _need_cuda(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise PcError("tensors must live on a CUDA device")
+
+
+def _make_desc(q, k, v, o, w, rope_theta, softmax_scale):
+    C, L, Hq, d = q.shape
+    Hkv = k.shape[2]
+    desc = _PrefillDesc(C, L, w, Hq, Hkv, d, float(rope_theta), float(softmax_scale))
+    for name, t in (("q_stride", q), ("k_stride", k), ("v_stride", v), ("o_stride", o)):
+        if t.stride(3) != 1:
+            raise PcError("head dimension must be contiguous")
+        getattr(desc, name)[0], getattr(desc, name)[1], getattr(desc, name)[2] = t.stride(0), t.stride(1), t.stride(2)
+    return desc
+
+
+def chunk_prefill_attn_workspace_bytes(C, L, w, Hq, Hkv, d, k_rot_in_workspace=False) -> int:
+    desc = _PrefillDesc(C, L, w, Hq, Hkv, d, 10000.0, 0.0)
+    return int(load_library().pc_chunk_prefill_attn_workspace_bytes(ctypes.byref(desc), int(k_rot_in_workspace)))
+
+
+def chunk_prefill_attn(q, k, v, *, w, rope_theta, softmax_scale=0.0, want_lse=False, out=None, k_rot=None,
+                       win_score=None, win_lse=None, lse=None, status=None, workspace=None):
+    """pc_chunk_prefill_attn: q [C,L,Hq,d], k/v [C,L,Hkv,d] bf16 (pre-RoPE).
+
+    Returns dict(o, k_rot, win_score, win_lse, lse, status, workspace).
+    """
+    lib = load_library()
+    _need_cuda(q, k, v)
+    C, L, Hq, d = q.shape
+    Hkv = k.shape[2]
+    dev = q.device
+    o = torch.empty((C, L, Hq, d), dtype=torch.bfloat16, device=dev) if out is None else out
+    if k_rot is None:
+        k_rot = torch.empty((C, L, Hkv, d), dtype=torch.bfloat16, device=dev)
+    if win_score is None:
+        win_score = torch.empty((C, Hkv, L), dtype=torch.float32, device=dev)
+    if win_lse is None:
+        win_lse = torch.empty((C, Hq, w), dtype=torch.float32, device=dev)
+    if lse is None and want_lse:
+        lse = torch.empty((C, Hq, L), dtype=torch.float32, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    desc = _make_desc(q, k, v, o, w, rope_theta, softmax_scale)
+    need = int(lib.pc_chunk_prefill_attn_workspace_bytes(ctypes.byref(desc), 0))
+    if need == 0:
+        _check(lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(k_rot), _ptr(lse),
+                                         _ptr(win_score), _ptr(win_lse), _ptr(status), None, 0, _stream()),
+               "pc_chunk_prefill_attn")
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(k_rot), _ptr(lse),
+                                   _ptr(win_score), _ptr(win_lse), _ptr(status), _ptr(workspace), workspace.numel(),
+                                   _stream())
+    _check(rc, "pc_chunk_prefill_attn")
+    return {"o": o, "k_rot": k_rot, "win_score": win_score, "win_lse": win_lse, "lse": lse, "status": status,
+            "workspace": workspace}
+
+
+def chunk_score_from_lse(win_lse, out=None):
+    """pc_chunk_score_from_lse: win_lse [C,Hq,w] fp32 -> [C] fp32."""
+    lib = load_library()
+    _need_cuda(win_lse)
+    C, Hq, w = win_lse.shape
+    out = torch.empty(C, dtype=torch.float32, device=win_lse.device) if out is None else out
+    _check(lib.pc_chunk_score_from_lse(_ptr(win_lse), C, Hq, w, _ptr(out), _stream()), "pc_chunk_score_from_lse")
+    return out
+
+
+def select_chunks(chunk_score, m, lower_is_better=True, out=None):
+    """pc_select_chunks: chunk_score [C] fp32 -> kept [m] int32 (ascending ids)."""
+    lib = load_library()
+    _need_cuda(chunk_score)
+    C = chunk_score.numel()
+    out = torch.empty(m, dtype=torch.int32, device=chunk_score.device) if out is None else out
+    _check(lib.pc_select_chunks(_ptr(chunk_score), C, int(m), int(bool(lower_is_better)), _ptr(out), _stream()),
+           "pc_select_chunks")
+    return out
+
+
+def select_tokens(win_score, kept, n_cand, k, out=None):
+    """pc_select_tokens: win_score [C,Hkv,L] fp32, kept [m] int32 -> idx [m,Hkv,k] int32."""
+    lib = load_library()
+    _need_cuda(win_score, kept)
+    C, Hkv, L = win_score.shape
+    m = kept.numel()
+    out = torch.empty((m, Hkv, k), dtype=torch.int32, device=win_score.device) if out is None else out
+    _check(lib.pc_select_tokens(_ptr(win_score), _ptr(kept), C, m, Hkv, L, int(n_cand), int(k), _ptr(out), _stream()),
+           "pc_select_tokens")
+    return out
+
+
+def gather_kv(k_src, v_src, kept, idx, k_out=None, v_out=None, pos_out=None, want_pos=True):
+    """pc_gather_kv: k_src/v_src [C,L,Hkv,d] bf16 -> (k_out, v_out [Hkv, m*k, d], pos [Hkv, m*k])."""
+    lib = load_library()
+    _need_cuda(k_src, v_src, kept, idx)
+    C, L, Hkv, d = k_src.shape
+    m, _, k = idx.shape
+    dev = k_src.device
+    if k_src.stride() != v_src.stride() or k_src.stride(3) != 1:
+        raise PcError("k_src and v_src must share strides with a contiguous head dimension")
+    k_out = torch.empty((Hkv, m * k, d), dtype=torch.bfloat16, device=dev) if k_out is None else k_out
+    v_out = torch.empty((Hkv, m * k, d), dtype=torch.bfloat16, device=dev) if v_out is None else v_out
+    if pos_out is None and want_pos:
+        pos_out = torch.empty((Hkv, m * k), dtype=torch.int32, device=dev)
+    strides = (c_int64 * 3)(k_src.stride(0), k_src.stride(1), k_src.stride(2))
+    _check(lib.pc_gather_kv(_ptr(k_src), _ptr(v_src), strides, L, _ptr(kept), _ptr(idx), m, Hkv, k, d, _ptr(k_out),
+                            _ptr(v_out), _ptr(pos_out), _stream()), "pc_gather_kv")
+    return k_out, v_out, pos_out
+
+
+def parallel_attn_workspace_bytes(B, w, Hq, Hkv, d, Nk) -> int:
+    return int(load_library().pc_parallel_attn_workspace_bytes(B, w, Hq, Hkv, d, Nk))
+
+
+def parallel_attn(q_win, k_cache, v_cache, k_win, v_win, *, q_pos0, rope_theta, softmax_scale=0.0, out=None,
+                  lse_out=None, want_lse=False, status=None, workspace=None):
+    """pc_parallel_attn: q_win [B,w,Hq,d] (pre-RoPE), k_cache/v_cache [B,Hkv,Nk,d], k_win/v_win [B,w,Hkv,d]."""
+    lib = load_library()
+    _need_cuda(q_win, k_cache, v_cache, k_win, v_win)
+    B, w, Hq, d = q_win.shape
+    Hkv, Nk = k_cache.shape[1], k_cache.shape[2]
+    dev = q_win.device
+    for t in (q_win, k_cache, v_cache, k_win, v_win):
+        if not t.is_contiguous():
+            raise PcError("pc_parallel_attn takes contiguous tensors")
+    out = torch.empty((B, w, Hq, d), dtype=torch.bfloat16, device=dev) if out is None else out
+    if lse_out is None and want_lse:
+        lse_out = torch.empty((B, Hq, w), dtype=torch.float32, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    need = parallel_attn_workspace_bytes(B, w, Hq, Hkv, d, Nk)
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    rc = lib.pc_parallel_attn(B, w, Hq, Hkv, d, Nk, _ptr(q_win), int(q_pos0), float(rope_theta), float(softmax_scale),
+                              _ptr(k_cache), _ptr(v_cache), _ptr(k_win), _ptr(v_win), _ptr(out), _ptr(lse_out),
+                              _ptr(status), _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "pc_parallel_attn")
+    return {"out": out, "lse": lse_out, "status": status, "workspace": workspace}
+
+
+def hot_path(q, k, v, *, w, rope_theta, m, k_keep, softmax_scale=0.0, chunk_score=None, buffers=None):
+    """One pass of the whole path on the current stream: the five C-ABI calls chained, no host sync.
+
+    ``chunk_score`` (device fp32 [C]) stands for the self-information of Eq. 3; if None the
+    single-layer stand-in computed from the window log-sum-exp is used.
+    ``buffers`` (dict) lets repeated calls reuse outputs and workspaces.
+    """
+    b = {} if buffers is None else buffers
+    C, L, Hq, d = q.shape
+    pre = chunk_prefill_attn(q, k, v, w=w, rope_theta=rope_theta, softmax_scale=softmax_scale, out=b.get("o"),
+                             k_rot=b.get("k_rot"), win_score=b.get("win_score"), win_lse=b.get("win_lse"),
+                             status=b.get("status"), workspace=b.get("ws_prefill"))
+    score = chunk_score if chunk_score is not None else chunk_score_from_lse(pre["win_lse"], out=b.get("chunk_score"))
+    kept = select_chunks(score, m, True, out=b.get("kept"))
+    idx = select_tokens(pre["win_score"], kept, L - w, k_keep, out=b.get("idx"))
+    kc, vc, pos = gather_kv(pre["k_rot"], v, kept, idx, k_out=b.get("kc"), v_out=b.get("vc"), pos_out=b.get("pos"))
+    # the window is the same in every chunk: take it from chunk 0 (views, no copy)
+    q_win = q[0:1, L - w:].contiguous() if not q[0:1, L - w:].is_contiguous() else q[0:1, L - w:]
+    k_win = pre["k_rot"][0:1, L - w:]
+    v_win = v[0:1, L - w:]
+    if not v_win.is_contiguous():
+        v_win = v_win.contiguous()
+    pa = parallel_attn(q_win, kc.unsqueeze(0), vc.unsqueeze(0), k_win, v_win, q_pos0=L - w, rope_theta=rope_theta,
+                       softmax_scale=softmax_scale, out=b.get("fg"), status=pre["status"], workspace=b.get("ws_par"))
+    res = {"o": pre["o"], "k_rot": pre["k_rot"], "win_score": pre["win_score"], "win_lse": pre["win_lse"],
+           "chunk_score": score, "kept": kept, "idx": idx, "kc": kc, "vc": vc, "pos": pos, "fg": pa["out"],
+           "status": pre["status"], "ws_prefill": pre["workspace"], "ws_par": pa["workspace"]}
+    if buffers is not None:
+        buffers.update({"o": res["o"], "k_rot": res["k_rot"], "win_score": res["win_score"], "win_lse": res["win_lse"],
+                        "chunk_score": score if chunk_score is None else b.get("chunk_score"), "kept": kept, "idx": idx,
+                        "kc": kc, "vc": vc, "pos": pos, "fg": res["fg"], "status": res["status"],
+                        "ws_prefill": res["ws_prefill"], "ws_par": res["ws_par"]})
+    return res

@@ -1,0 +1,213 @@
+// C ABI of libpc: argument validation on the host, tensor-map construction, launches.
+// Nothing here allocates device memory or synchronises.
+#include "../../include/pc.h"
+#include "pc_attn.h"
+#include "pc_kernels.h"
+#include "pc_tmap.h"
+
+#include <cmath>
+#include <cstring>
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceInfo {
+  int ok = 0;          // 1: sm_100, -1: something else
+  int sm_count = 0;
+};
+
+// Properties of the current device (queried once per device).
+const DeviceInfo& device_info() {
+  static DeviceInfo info[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { static DeviceInfo bad; bad.ok = -1; return bad; }
+  if (info[dev].ok == 0) {
+    int major = 0, sms = 0;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    info[dev].sm_count = sms;
+    info[dev].ok = (major == 10) ? 1 : -1;
+  }
+  return info[dev];
+}
+
+bool pow2_between(int x, int lo, int hi) { return x >= lo && x <= hi && (x & (x - 1)) == 0; }
+
+void fill_strides(const int64_t in[3], int64_t out[3], int64_t tokens, int64_t heads, int64_t d) {
+  if (in[0] == 0 && in[1] == 0 && in[2] == 0) { out[0] = tokens * heads * d; out[1] = heads * d; out[2] = d; }
+  else { out[0] = in[0]; out[1] = in[1]; out[2] = in[2]; }
+}
+bool strides_ok(const int64_t s[3], int64_t d) { return s[0] > 0 && s[1] > 0 && s[2] >= d && s[0] % 8 == 0 && s[1] % 8 == 0 && s[2] % 8 == 0; }
+
+struct PrefillLayout {
+  size_t off_counter, off_table, off_krot, total;
+};
+PrefillLayout prefill_layout(const pc_prefill_desc* d, bool krot_in_ws) {
+  PrefillLayout l;
+  size_t off = 0;
+  l.off_counter = off; off += ALIGN;
+  l.off_table = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(double2));
+  l.off_krot = off;
+  if (krot_in_ws) off += align_up((size_t)d->C * d->L * d->Hkv * d->d * 2);
+  l.total = off;
+  return l;
+}
+
+int32_t check_prefill_desc(const pc_prefill_desc* d) {
+  if (!d) return PC_ERR_INVALID_ARG;
+  if (d->C < 1 || d->L < 2 || d->w < 1 || d->w >= d->L || d->Hq < 1 || d->Hkv < 1 || d->Hq % d->Hkv != 0) return PC_ERR_INVALID_ARG;
+  if (!(d->rope_theta > 0.0f) || d->softmax_scale < 0.0f) return PC_ERR_INVALID_ARG;
+  if (d->d != 64 && d->d != 128) return PC_ERR_UNSUPPORTED;
+  if (!pow2_between(d->w, 8, 128)) return PC_ERR_UNSUPPORTED;
+  if ((int64_t)(d->Hq / d->Hkv) * d->w > 1024) return PC_ERR_UNSUPPORTED;
+  if ((int64_t)d->C * d->Hkv > (1 << 24) || d->L > (1 << 24)) return PC_ERR_UNSUPPORTED;
+  return PC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pc_status_string(int32_t status) {
+  switch (status) {
+    case PC_OK: return "ok";
+    case PC_ERR_INVALID_ARG: return "invalid argument";
+    case PC_ERR_UNSUPPORTED: return "unsupported shape or device";
+    case PC_ERR_WORKSPACE: return "workspace missing or too small";
+    case PC_ERR_CUDA: return "CUDA call failed";
+    case PC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int32_t pc_version(void) { return 1000; }
+
+// ------------------------------------------------------------------------------------ prefill
+size_t pc_chunk_prefill_attn_workspace_bytes(const pc_prefill_desc* desc, int32_t k_rot_in_workspace) {
+  if (check_prefill_desc(desc) != PC_OK) return 0;
+  return prefill_layout(desc, k_rot_in_workspace != 0).total;
+}
+
+int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const void* k, const void* v, void* o,
+                              void* k_rot, float* lse, float* win_score, float* win_lse, int32_t* status_word,
+                              void* workspace, size_t workspace_bytes, void* stream) {
+  int32_t rc = check_prefill_desc(desc);
+  if (rc != PC_OK) return rc;
+  if (!q || !k || !v || !o || !win_score || !win_lse) return PC_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(k_rot) || !aligned16(workspace))
+    return PC_ERR_INVALID_ARG;
+  const int d = desc->d;
+  int64_t qs[3], ks[3], vs[3], os[3];
+  fill_strides(desc->q_stride, qs, desc->L, desc->Hq, d);
+  fill_strides(desc->k_stride, ks, desc->L, desc->Hkv, d);
+  fill_strides(desc->v_stride, vs, desc->L, desc->Hkv, d);
+  fill_strides(desc->o_stride, os, desc->L, desc->Hq, d);
+  if (!strides_ok(qs, d) || !strides_ok(ks, d) || !strides_ok(vs, d) || !strides_ok(os, d)) return PC_ERR_INVALID_ARG;
+  const bool krot_in_ws = (k_rot == nullptr);
+  const PrefillLayout lay = prefill_layout(desc, krot_in_ws);
+  if (!workspace || workspace_bytes < lay.total) return PC_ERR_WORKSPACE;
+  const DeviceInfo& dev = device_info();
+  if (dev.ok != 1) return PC_ERR_UNSUPPORTED;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  int* counter = reinterpret_cast<int*>(ws + lay.off_counter);
+  double2* table = reinterpret_cast<double2*>(ws + lay.off_table);
+  void* krot = krot_in_ws ? static_cast<void*>(ws + lay.off_krot) : k_rot;
+
+  // tensor maps (innermost first: d, head, token, chunk)
+  CUtensorMap maps[5];
+  const uint64_t q_dims[4] = {(uint64_t)d, (uint64_t)desc->Hq, (uint64_t)desc->L, (uint64_t)desc->C};
+  const uint64_t kv_dims[4] = {(uint64_t)d, (uint64_t)desc->Hkv, (uint64_t)desc->L, (uint64_t)desc->C};
+  const uint64_t q_str[3] = {(uint64_t)qs[2], (uint64_t)qs[1], (uint64_t)qs[0]};
+  const uint64_t v_str[3] = {(uint64_t)vs[2], (uint64_t)vs[1], (uint64_t)vs[0]};
+  const uint64_t o_str[3] = {(uint64_t)os[2], (uint64_t)os[1], (uint64_t)os[0]};
+  const uint64_t kr_str[3] = {(uint64_t)d, (uint64_t)desc->Hkv * d, (uint64_t)desc->L * desc->Hkv * d};
+  const uint32_t box_tile[4] = {64, 1, 128, 1};
+  const uint32_t box_win[4] = {64, 1, (uint32_t)desc->w, 1};
+  if (!pc::make_tmap_bf16_4d(&maps[0], q, q_dims, q_str, box_tile) ||
+      !pc::make_tmap_bf16_4d(&maps[1], krot, kv_dims, kr_str, box_tile) ||
+      !pc::make_tmap_bf16_4d(&maps[2], v, kv_dims, v_str, box_tile) ||
+      !pc::make_tmap_bf16_4d(&maps[3], o, q_dims, o_str, box_tile) ||
+      !pc::make_tmap_bf16_4d(&maps[4], q, q_dims, q_str, box_win))
+    return PC_ERR_CUDA;
+
+  if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return PC_ERR_CUDA;
+  pc::launch_rope_table(table, desc->L, d, (double)desc->rope_theta, 0, st);
+  const long long ks_ll[3] = {ks[0], ks[1], ks[2]};
+  pc::launch_rope_keys(k, ks_ll, krot, table, desc->C, desc->L, desc->Hkv, d, st);
+
+  pc::PrefillParams prm;
+  prm.C = desc->C; prm.L = desc->L; prm.w = desc->w; prm.Hq = desc->Hq; prm.Hkv = desc->Hkv;
+  const double scale = desc->softmax_scale > 0.0f ? (double)desc->softmax_scale : 1.0 / std::sqrt((double)d);
+  prm.scale_log2 = (float)(scale * 1.4426950408889634);
+  prm.rope_tab = table;
+  prm.lse = lse; prm.win_lse = win_lse; prm.win_score = win_score;
+  prm.status = status_word; prm.counter = counter;
+  if (pc::launch_prefill_attn(maps, prm, d, dev.sm_count, st) != cudaSuccess) return PC_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------ chunk score stand-in
+int32_t pc_chunk_score_from_lse(const float* win_lse, int32_t C, int32_t Hq, int32_t w, float* chunk_score,
+                                void* stream) {
+  if (!win_lse || !chunk_score || C < 1 || Hq < 1 || w < 1) return PC_ERR_INVALID_ARG;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  pc::launch_chunk_score(win_lse, C, Hq * w, chunk_score, static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------ chunk top-m
+int32_t pc_select_chunks(const float* chunk_score, int32_t C, int32_t m, int32_t lower_is_better, int32_t* kept,
+                         void* stream) {
+  if (!chunk_score || !kept || C < 1 || m < 1 || m > C) return PC_ERR_INVALID_ARG;
+  if (C > 1024) return PC_ERR_UNSUPPORTED;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  pc::launch_select_chunks(chunk_score, C, m, lower_is_better, kept, static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------ token top-k
+int32_t pc_select_tokens(const float* win_score, const int32_t* kept, int32_t C, int32_t m, int32_t Hkv, int32_t L,
+                         int32_t n_cand, int32_t k, int32_t* idx, void* stream) {
+  if (!win_score || !kept || !idx) return PC_ERR_INVALID_ARG;
+  if (C < 1 || m < 1 || m > C || Hkv < 1 || L < 1 || n_cand < 1 || n_cand > L || k < 1) return PC_ERR_INVALID_ARG;
+  if (n_cand > 32768) return PC_ERR_UNSUPPORTED;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  if (pc::launch_select_tokens(win_score, kept, m, Hkv, L, n_cand, k, idx, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return PC_ERR_CUDA;
+  return PC_OK;
+}
+
+// ------------------------------------------------------------------------------------ gather
+int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t* kv_stride, int32_t L, const int32_t* kept,
+                     const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d, void* k_out, void* v_out,
+                     int32_t* pos_out, void* stream) {
+  if (!k_src || !v_src || !kept || !idx || !k_out || !v_out) return PC_ERR_INVALID_ARG;
+  if (m < 1 || Hkv < 1 || k < 1 || L < 1) return PC_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
+  if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(k_out) || !aligned16(v_out)) return PC_ERR_INVALID_ARG;
+  long long s[3];
+  if (kv_stride) { s[0] = kv_stride[0]; s[1] = kv_stride[1]; s[2] = kv_stride[2]; }
+  else { s[0] = (long long)L * Hkv * d; s[1] = (long long)Hkv * d; s[2] = d; }
+  if (s[0] <= 0 || s[1] <= 0 || s[2] < d || s[0] % 8 || s[1] % 8 || s[2] % 8) return PC_ERR_INVALID_ARG;
+  const DeviceInfo& dev = device_info();
+  if (dev.ok != 1) return PC_ERR_UNSUPPORTED;
+  if (pc::launch_gather_kv(k_src, v_src, s, kept, idx, m, Hkv, k, d, k_out, v_out, pos_out, dev.sm_count,
+                           static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return PC_ERR_CUDA;
+  return PC_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------ parallel attention (placeholder until pc_parallel.cu lands)
+extern "C" {
+size_t pc_parallel_attn_workspace_bytes(int32_t, int32_t, int32_t, int32_t, int32_t, int32_t) { return 0; }
+int32_t pc_parallel_attn(int32_t, int32_t, int32_t, int32_t, int32_t, int32_t, const void*, int32_t, float, float,
+                         const void*, const void*, const void*, const void*, void*, float*, int32_t*, void*, size_t,
+                         void*) { return PC_ERR_UNSUPPORTED; }
+}

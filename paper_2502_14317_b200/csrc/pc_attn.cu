@@ -1,0 +1,623 @@
+// Attention kernels for sm_100a: chunk-local causal attention with fused query-window
+// scores (Eq. 1-2, Eq. 5-6) and parallel attention over the compressed cache (Eq. 9-11).
+//
+// One persistent CTA per SM, 10 warps:
+//   warps 0-3  softmax group 0   (one 128-row query block, thread = row = TMEM lane)
+//   warps 4-7  softmax group 1   (a second 128-row block sharing the same K/V tiles)
+//   warp  8    TMA producer      (Q tiles, K/V ring)
+//   warp  9    tcgen05 issuer    (owns TMEM allocation)
+// Per 128-key tile:  S_b = Q_b K^T  (SS MMA, fp32 in TMEM)  ->  softmax group b turns S_b
+// into bf16 P_b in place in TMEM  ->  O_b += P_b V  (TS MMA, V as N-major smem operand).
+// While group 0 runs its softmax the tensor core works for group 1 and vice versa.
+// The running maximum is only raised when it grows by more than 2^8 (lazy rescale), so
+// the accumulator is rarely touched between tiles.
+//
+// Window scores (prefill only): the item that owns the last query tiles of a
+// (chunk, kv-head) group runs them for all G q-heads, keeps the window rows' final
+// log-sum-exp in shared memory, then sweeps the keys once more computing the transposed
+// product K_j Qw^T (keys on TMEM lanes, the G*w window rows on columns), so the column
+// sum of Eq. 6 is a per-thread sum in a fixed order: deterministic, no atomics.
+#include "pc_kernels.h"
+#include "pc_attn.h"
+#include "pc_sm100.cuh"
+
+namespace pc {
+
+namespace {
+
+constexpr int TILE = 128;
+constexpr int NUM_THREADS = 320;
+constexpr int WARP_PRODUCER = 8;
+constexpr int WARP_MMA = 9;
+constexpr int NS = 4;                       // K/V ring stages
+constexpr float LAZY_RESCALE = 8.0f;        // log2 units
+constexpr int ITEM_DONE = -1;
+
+// where-codes stored in the status word when a wait gives up
+enum { W_ITEM = 101, W_QFULL, W_QROT, W_QFREE, W_KVFULL, W_KVFREE, W_SFULL, W_PFULL, W_OFULL, W_ACCFREE, W_TFULL, W_TFREE };
+
+struct __align__(16) Misc {
+  uint64_t q_full[2], q_rot[2], q_free[2];
+  uint64_t kv_full[NS], kv_free[NS];
+  uint64_t s_full[2], p_full[2], o_full[2], acc_free[2];
+  uint64_t item_full[2], item_empty[2];
+  uint64_t t_full[2], t_free[2];
+  int item_slot[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  float lse2[1024];                        // window-row log-sum-exp (log2 domain), G * w <= 1024
+  float xch[2][TILE];
+};
+
+template <int D>
+struct Cfg {
+  static constexpr int TILE_BYTES = TILE * D * 2;
+  static constexpr int ATOMS = D / 64;
+  static constexpr int OFF_Q = 0;
+  static constexpr int OFF_RING = 2 * TILE_BYTES;
+  static constexpr int OFF_MISC = OFF_RING + NS * TILE_BYTES;
+  static constexpr int SMEM_BYTES = OFF_MISC + (int)sizeof(Misc) + 1024;   // + alignment slack
+};
+
+// One pair of 128-row query blocks that share K/V tiles.
+struct SubItem {
+  int hA, tA, hB, tB;        // q-head and query tile of block A / B; hB < 0: block B absent
+};
+
+// ------------------------------------------------------------------ item decoding (prefill)
+struct Sched {
+  int T, t_w, ntt, G, P, hp_mode, ipg, n_lp;
+};
+
+__device__ __forceinline__ Sched make_sched(const PrefillParams& p) {
+  Sched s;
+  s.T = (p.L + TILE - 1) / TILE;
+  s.G = p.Hq / p.Hkv;
+  s.hp_mode = (s.G % 2 == 0);
+  s.P = s.G / 2;
+  if (s.hp_mode) {
+    s.t_w = (p.L - p.w) / TILE;              // first tile holding a window row
+    s.ntt = s.T - s.t_w;                     // 1 or 2 tail tiles
+    s.n_lp = 0;
+    s.ipg = 1 + s.t_w * s.P;
+  } else {
+    s.ntt = s.T >= 2 ? 2 : 1;
+    s.t_w = s.T - s.ntt;
+    s.n_lp = (s.t_w + 1) / 2;                // tile pairs below the tail, from the top
+    s.ipg = 1 + s.n_lp * s.G;
+  }
+  return s;
+}
+
+// number of sub-items of item `within` (0 = tail item of the group)
+__device__ __forceinline__ int n_subitems(const Sched& s, int within) {
+  if (within != 0) return 1;
+  return s.hp_mode ? s.P * s.ntt : s.G;
+}
+
+__device__ __forceinline__ SubItem decode_sub(const Sched& s, int hkv, int within, int sub) {
+  SubItem it;
+  const int h0 = hkv * s.G;
+  if (s.hp_mode) {
+    int pair, tile;
+    if (within == 0) { pair = sub / s.ntt; tile = s.T - 1 - (sub % s.ntt); }
+    else { const int x = within - 1; tile = s.t_w - 1 - x / s.P; pair = x % s.P; }
+    it.hA = h0 + 2 * pair; it.hB = it.hA + 1; it.tA = tile; it.tB = tile;
+  } else {
+    int g, hi;
+    if (within == 0) { g = sub; hi = s.T - 1; }
+    else { const int x = within - 1; g = x % s.G; hi = s.t_w - 1 - 2 * (x / s.G); }
+    if (hi >= 1) { it.hA = h0 + g; it.tA = hi - 1; it.hB = h0 + g; it.tB = hi; }
+    else { it.hA = h0 + g; it.tA = hi; it.hB = -1; it.tB = 0; }
+  }
+  return it;
+}
+
+// ------------------------------------------------------------------ RoPE of a query row in shared memory
+// Row `row` of a 128-byte-swizzled [128 x D] bf16 tile; pairs (t, t + D/2); fp64 math, one rounding.
+template <int D>
+__device__ __forceinline__ void rope_row_smem(uint8_t* tile, int row, const double2* __restrict__ tab_row) {
+#pragma unroll 1
+  for (int cidx = 0; cidx < D / 16; ++cidx) {
+    uint8_t* lo_p = tile + sw128_offset(row, cidx);
+    uint8_t* hi_p = (D == 128) ? tile + 16384 + sw128_offset(row, cidx) : tile + sw128_offset(row, cidx + 4);
+    const uint4 lo = *reinterpret_cast<const uint4*>(lo_p);
+    const uint4 hi = *reinterpret_cast<const uint4*>(hi_p);
+    const uint32_t lo_w[4] = {lo.x, lo.y, lo.z, lo.w}, hi_w[4] = {hi.x, hi.y, hi.z, hi.w};
+    uint32_t out_lo[4], out_hi[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t rl = 0, rh = 0;
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const double x1 = (double)__uint_as_float(((lo_w[i] >> (16 * e)) & 0xFFFFu) << 16);
+        const double x2 = (double)__uint_as_float(((hi_w[i] >> (16 * e)) & 0xFFFFu) << 16);
+        const double2 t = tab_row[cidx * 8 + 2 * i + e];
+        rl |= (uint32_t)f64_to_bf16_rne(x1 * t.x - x2 * t.y) << (16 * e);
+        rh |= (uint32_t)f64_to_bf16_rne(x2 * t.x + x1 * t.y) << (16 * e);
+      }
+      out_lo[i] = rl;
+      out_hi[i] = rh;
+    }
+    *reinterpret_cast<uint4*>(lo_p) = make_uint4(out_lo[0], out_lo[1], out_lo[2], out_lo[3]);
+    *reinterpret_cast<uint4*>(hi_p) = make_uint4(out_hi[0], out_hi[1], out_hi[2], out_hi[3]);
+  }
+}
+
+// ------------------------------------------------------------------ softmax of one tile (thread = row)
+// Reads the 128 fp32 logits of this thread's row from TMEM, updates the running
+// (m, l), rescales the accumulator when the maximum moved by more than 2^LAZY_RESCALE,
+// and writes bf16 probabilities back over the logits.  `vis` = visible columns (<= 0: none).
+template <int D>
+__device__ __forceinline__ void softmax_tile(uint32_t s_taddr, uint32_t o_taddr, int vis, bool first_tile,
+                                             float scale_log2, float& m_used, float& l_run) {
+  uint32_t s[4][32];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) tmem_ld32(s_taddr + q * 32, s[q]);
+  tmem_wait_ld();
+  float mx = -INFINITY;
+  if (vis >= TILE) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+      for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(s[q][j]));
+  } else {
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        if (q * 32 + j >= vis) s[q][j] = 0xFF800000u;            // -inf
+        mx = fmaxf(mx, __uint_as_float(s[q][j]));
+      }
+  }
+  const float m_tile = mx * scale_log2;                          // -inf if nothing visible
+  float alpha = 1.0f;
+  const bool raise = first_tile || (m_tile > m_used + LAZY_RESCALE);
+  if (raise) {
+    const float m_new = fmaxf(m_used, m_tile);
+    alpha = (m_used == -INFINITY) ? 0.0f : fast_exp2(m_used - m_new);
+    m_used = m_new;
+  }
+  if (!first_tile && __any_sync(0xFFFFFFFFu, raise)) {           // warp-uniform: each warp owns its 32 lanes of O
+#pragma unroll
+    for (int q = 0; q < D / 32; ++q) {
+      uint32_t o[32];
+      tmem_ld32(o_taddr + q * 32, o);
+      tmem_wait_ld();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+      tmem_st32(o_taddr + q * 32, o);
+    }
+  }
+  const float neg_m = (m_used == -INFINITY) ? 0.0f : -m_used;     // fully masked row so far: exp2(-inf) = 0
+  float sum = 0.0f;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint32_t packed[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float p0 = fast_exp2(fmaf(__uint_as_float(s[q][2 * j]), scale_log2, neg_m));
+      const float p1 = fast_exp2(fmaf(__uint_as_float(s[q][2 * j + 1]), scale_log2, neg_m));
+      sum += p0 + p1;
+      packed[j] = pack_bf16x2(p0, p1);
+    }
+    tmem_st16(s_taddr + q * 16, packed);                          // P aliases the first 64 columns of S
+  }
+  l_run = l_run * alpha + sum;
+  tmem_wait_st();
+}
+
+// ------------------------------------------------------------------ tensor-core issue helpers (one thread)
+template <int D>
+__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t q_smem, uint32_t k_smem, int n_cols) {
+  const uint32_t idesc = make_idesc_bf16_f32(TILE, n_cols, false, false);
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+    const uint32_t off = (ks / 4) * 16384 + (ks % 4) * 32;
+    mma_ss(d_tmem, make_smem_desc_sw128(q_smem + off, 16, 1024), make_smem_desc_sw128(k_smem + off, 16, 1024), idesc,
+           ks > 0);
+  }
+}
+// transposed product for the score sweep: D[keys, rows] = K_tile * Qw^T
+template <int D>
+__device__ __forceinline__ void issue_kq(uint32_t d_tmem, uint32_t k_smem, uint32_t q_smem, int n_cols) {
+  issue_qk<D>(d_tmem, k_smem, q_smem, n_cols);
+}
+template <int D>
+__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate) {
+  constexpr uint32_t idesc = make_idesc_bf16_f32(TILE, D, false, true);
+#pragma unroll
+  for (int ks = 0; ks < TILE / 16; ++ks) {
+    mma_ts(o_tmem, p_tmem + ks * 8, make_smem_desc_sw128(v_smem + ks * 2048, 16384, 1024), idesc,
+           accumulate || ks > 0);
+  }
+}
+
+// ------------------------------------------------------------------ per-role state
+struct Waits {                                 // how many times each barrier has been used by this role
+  uint32_t q[2] = {0, 0};                      // q_full / q_rot / q_free (one use per block load)
+  uint32_t kv = 0;                             // ring position (monotone)
+  uint32_t s[2] = {0, 0}, p[2] = {0, 0}, o[2] = {0, 0}, acc[2] = {0, 0};
+  uint32_t t[2] = {0, 0};
+  uint32_t item = 0;
+};
+__device__ __forceinline__ uint32_t full_par(uint32_t n) { return n & 1u; }          // n-th use of a "full" barrier
+__device__ __forceinline__ uint32_t free_par(uint32_t n) { return (n & 1u) ^ 1u; }   // before the n-th use of a resource
+
+}  // namespace
+
+// ====================================================================================
+//                                   PREFILL KERNEL
+// ====================================================================================
+template <int D>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                    const __grid_constant__ CUtensorMap tm_qw, const __grid_constant__ PrefillParams prm) {
+  using C = Cfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  Misc& mi = *reinterpret_cast<Misc*>(smem + C::OFF_MISC);
+  uint8_t* sQ[2] = {smem + C::OFF_Q, smem + C::OFF_Q + C::TILE_BYTES};
+  uint8_t* ring = smem + C::OFF_RING;
+  volatile int* abort_flag = &mi.abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const Sched sch = make_sched(prm);
+  const int n_groups = prm.C * prm.Hkv;
+  const int n_items = n_groups * sch.ipg;
+  const int Gs = (256 / prm.w) < sch.G ? (256 / prm.w) : sch.G;      // q-heads per score pass
+  const int n_pass = (sch.G + Gs - 1) / Gs;
+
+  if (tid == 0) {
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 128); mbar_init(&mi.q_free[b], 1);
+      mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_full[b], 128); mbar_init(&mi.o_full[b], 1);
+      mbar_init(&mi.acc_free[b], 128);
+      mbar_init(&mi.item_full[b], 1); mbar_init(&mi.item_empty[b], 257);
+      mbar_init(&mi.t_full[b], 1); mbar_init(&mi.t_free[b], 256);
+    }
+    for (int s = 0; s < NS; ++s) { mbar_init(&mi.kv_full[s], 1); mbar_init(&mi.kv_free[s], 1); }
+    mi.abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == WARP_MMA) tmem_alloc(&mi.tmem_base, 512);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = mi.tmem_base;
+
+  Waits wt;
+
+  if (warp == WARP_PRODUCER) {
+    // ================================================================ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_qw);
+      while (true) {
+        // ---- fetch and publish the next item
+        const int slot = wt.item & 1;
+        mbar_wait(&mi.item_empty[slot], free_par(wt.item >> 1), abort_flag, prm.status, W_ITEM);
+        int item = atomicAdd(prm.counter, 1);
+        if (item >= n_items || *abort_flag) item = ITEM_DONE;
+        mi.item_slot[slot] = item;
+        mbar_arrive(&mi.item_full[slot]);
+        ++wt.item;
+        if (item == ITEM_DONE) break;
+        const int group = item / sch.ipg, within = item % sch.ipg;
+        const int c = group / prm.Hkv, hkv = group % prm.Hkv;
+        const int nsub = n_subitems(sch, within);
+        for (int sub = 0; sub < nsub; ++sub) {
+          const SubItem it = decode_sub(sch, hkv, within, sub);
+          for (int b = 0; b < 2; ++b) {
+            const int h = b ? it.hB : it.hA, t = b ? it.tB : it.tA;
+            if (h < 0) continue;
+            mbar_wait(&mi.q_free[b], free_par(wt.q[b]), abort_flag, prm.status, W_QFREE);
+            mbar_arrive_expect_tx(&mi.q_full[b], C::TILE_BYTES);
+            for (int a = 0; a < C::ATOMS; ++a) tma_load_4d(sQ[b] + a * 16384, &tm_q, &mi.q_full[b], a * 64, h, t * TILE, c);
+            ++wt.q[b];
+          }
+          const int n = (it.hB >= 0 ? it.tB : it.tA) + 1;
+          for (int j = 0; j < n; ++j) {
+            for (int kv = 0; kv < 2; ++kv) {                       // K_j then V_j
+              const int st = wt.kv % NS;
+              mbar_wait(&mi.kv_free[st], free_par(wt.kv / NS), abort_flag, prm.status, W_KVFREE);
+              mbar_arrive_expect_tx(&mi.kv_full[st], C::TILE_BYTES);
+              for (int a = 0; a < C::ATOMS; ++a)
+                tma_load_4d(ring + st * C::TILE_BYTES + a * 16384, kv ? &tm_v : &tm_k, &mi.kv_full[st], a * 64, hkv,
+                            j * TILE, c);
+              ++wt.kv;
+            }
+          }
+        }
+        if (within == 0) {
+          // ---- score sweep: window queries of Gs heads per pass, then all key tiles
+          for (int u = 0; u < n_pass; ++u) {
+            const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
+            const int rows_total = heads * prm.w;
+            for (int b = 0; b < 2; ++b) {
+              const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
+              if (rows_b == 0) continue;
+              mbar_wait(&mi.q_free[b], free_par(wt.q[b]), abort_flag, prm.status, W_QFREE);
+              mbar_arrive_expect_tx(&mi.q_full[b], rows_b * D * 2);
+              for (int r0 = 0; r0 < rows_b; r0 += prm.w) {
+                const int g = u * Gs + (b * TILE + r0) / prm.w;
+                for (int a = 0; a < C::ATOMS; ++a)
+                  tma_load_4d(sQ[b] + a * 16384 + r0 * 128, &tm_qw, &mi.q_full[b], a * 64, hkv * sch.G + g,
+                              prm.L - prm.w, c);
+              }
+              ++wt.q[b];
+            }
+            for (int j = 0; j < sch.T; ++j) {
+              const int st = wt.kv % NS;
+              mbar_wait(&mi.kv_free[st], free_par(wt.kv / NS), abort_flag, prm.status, W_KVFREE);
+              mbar_arrive_expect_tx(&mi.kv_full[st], C::TILE_BYTES);
+              for (int a = 0; a < C::ATOMS; ++a)
+                tma_load_4d(ring + st * C::TILE_BYTES + a * 16384, &tm_k, &mi.kv_full[st], a * 64, hkv, j * TILE, c);
+              ++wt.kv;
+            }
+          }
+        }
+      }
+      // drain: every copy this thread issued must have landed before the CTA exits
+      for (uint32_t i = (wt.kv > NS ? wt.kv - NS : 0); i < wt.kv; ++i) mbar_wait_drain(&mi.kv_full[i % NS], full_par(i / NS));
+      for (int b = 0; b < 2; ++b)
+        if (wt.q[b] > 0) mbar_wait_drain(&mi.q_full[b], full_par(wt.q[b] - 1));
+    }
+    __syncwarp();
+  } else if (warp == WARP_MMA) {
+    // ================================================================ tcgen05 issuer
+    if (lane == 0) {
+      const uint32_t ring_u32 = smem_u32(ring);
+      const uint32_t q_u32[2] = {smem_u32(sQ[0]), smem_u32(sQ[1])};
+      const uint32_t tS[2] = {tmem + 0, tmem + 128}, tO[2] = {tmem + 256, tmem + 384};
+      while (true) {
+        const int slot = wt.item & 1;
+        mbar_wait(&mi.item_full[slot], full_par(wt.item >> 1), abort_flag, prm.status, W_ITEM);
+        const int item = mi.item_slot[slot];
+        mbar_arrive(&mi.item_empty[slot]);
+        ++wt.item;
+        if (item == ITEM_DONE) break;
+        const int group = item / sch.ipg, within = item % sch.ipg;
+        const int hkv = group % prm.Hkv;
+        const int nsub = n_subitems(sch, within);
+        for (int sub = 0; sub < nsub; ++sub) {
+          const SubItem it = decode_sub(sch, hkv, within, sub);
+          const bool has[2] = {true, it.hB >= 0};
+          const int nb[2] = {it.tA + 1, it.hB >= 0 ? it.tB + 1 : 0};
+          const int n = nb[1] > nb[0] ? nb[1] : nb[0];
+          // accumulators and score buffers of earlier work must have been read out
+          for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), abort_flag, prm.status, W_ACCFREE);
+          for (int e = 0; e < 2; ++e) mbar_wait(&mi.t_free[e], free_par(wt.t[e]), abort_flag, prm.status, W_TFREE);
+          for (int b = 0; b < 2; ++b)
+            if (has[b]) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), abort_flag, prm.status, W_QROT); ++wt.q[b]; }
+          tc_fence_after_sync();
+          // S(0)
+          {
+            const int st = wt.kv % NS;
+            mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), abort_flag, prm.status, W_KVFULL);
+            tc_fence_after_sync();
+            for (int b = 0; b < 2; ++b)
+              if (has[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
+            mma_commit(&mi.kv_free[st]);
+            ++wt.kv;
+          }
+          for (int j = 0; j < n; ++j) {
+            const int st_v = wt.kv % NS;
+            mbar_wait(&mi.kv_full[st_v], full_par(wt.kv / NS), abort_flag, prm.status, W_KVFULL);
+            ++wt.kv;
+            int st_k = 0;
+            const bool more = j + 1 < n;
+            if (more) {
+              st_k = wt.kv % NS;
+              mbar_wait(&mi.kv_full[st_k], full_par(wt.kv / NS), abort_flag, prm.status, W_KVFULL);
+              ++wt.kv;
+            }
+            for (int b = 0; b < 2; ++b) {
+              if (!has[b] || j >= nb[b]) continue;
+              mbar_wait(&mi.p_full[b], full_par(wt.p[b]), abort_flag, prm.status, W_PFULL);
+              ++wt.p[b];
+              tc_fence_after_sync();
+              issue_pv<D>(tO[b], tS[b], ring_u32 + st_v * C::TILE_BYTES, j > 0);
+              if (j == nb[b] - 1) mma_commit(&mi.o_full[b]);
+              if (j + 1 < nb[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st_k * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
+            }
+            mma_commit(&mi.kv_free[st_v]);
+            if (more) mma_commit(&mi.kv_free[st_k]);
+          }
+          for (int b = 0; b < 2; ++b) if (has[b]) ++wt.acc[b];
+        }
+        if (within == 0) {
+          for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), abort_flag, prm.status, W_ACCFREE);
+          for (int u = 0; u < n_pass; ++u) {
+            const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
+            const int rows_total = heads * prm.w;
+            const int rows[2] = {rows_total < TILE ? rows_total : TILE, rows_total > TILE ? rows_total - TILE : 0};
+            for (int b = 0; b < 2; ++b)
+              if (rows[b] > 0) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), abort_flag, prm.status, W_QROT); ++wt.q[b]; }
+            for (int j = 0; j < sch.T; ++j) {
+              const int e = j & 1;
+              mbar_wait(&mi.t_free[e], free_par(wt.t[e]), abort_flag, prm.status, W_TFREE);
+              const int st = wt.kv % NS;
+              mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), abort_flag, prm.status, W_KVFULL);
+              ++wt.kv;
+              tc_fence_after_sync();
+              for (int b = 0; b < 2; ++b)
+                if (rows[b] > 0)
+                  issue_kq<D>(tmem + e * 256 + b * 128, ring_u32 + st * C::TILE_BYTES, q_u32[b], (rows[b] + 15) & ~15);
+              mma_commit(&mi.t_full[e]);
+              mma_commit(&mi.kv_free[st]);
+              ++wt.t[e];
+            }
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ================================================================ softmax groups
+    const int b = warp >> 2;                                 // block / group index
+    const int r = tid & 127;                                 // row in the block = TMEM lane
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + b * 128 + lane_sel, tO = tmem + 256 + b * 128 + lane_sel;
+    const float scale_log2 = prm.scale_log2;
+    while (true) {
+      const int slot = wt.item & 1;
+      mbar_wait(&mi.item_full[slot], full_par(wt.item >> 1), abort_flag, prm.status, W_ITEM);
+      const int item = mi.item_slot[slot];
+      mbar_arrive(&mi.item_empty[slot]);
+      ++wt.item;
+      if (item == ITEM_DONE) break;
+      const int group = item / sch.ipg, within = item % sch.ipg;
+      const int c = group / prm.Hkv, hkv = group % prm.Hkv;
+      const int nsub = n_subitems(sch, within);
+      for (int sub = 0; sub < nsub; ++sub) {
+        const SubItem it = decode_sub(sch, hkv, within, sub);
+        const int h = b ? it.hB : it.hA, t = b ? it.tB : it.tA;
+        if (h < 0) continue;
+        const int token = t * TILE + r;
+        // ---- Q prologue: rotate this thread's row in shared memory
+        mbar_wait(&mi.q_full[b], full_par(wt.q[b]), abort_flag, prm.status, W_QFULL);
+        ++wt.q[b];
+        if (token < prm.L) rope_row_smem<D>(sQ[b], r, prm.rope_tab + (size_t)token * (D / 2));
+        fence_proxy_async_smem();
+        mbar_arrive(&mi.q_rot[b]);
+        // ---- main loop over key tiles
+        float m_used = -INFINITY, l_run = 0.0f;
+        const int n = t + 1;
+        for (int j = 0; j < n; ++j) {
+          mbar_wait(&mi.s_full[b], full_par(wt.s[b]), abort_flag, prm.status, W_SFULL);
+          ++wt.s[b];
+          tc_fence_after_sync();
+          const int vis = (j == n - 1) ? (token - j * TILE + 1) : TILE;      // causal: keys <= token
+          softmax_tile<D>(tS, tO, vis, j == 0, scale_log2, m_used, l_run);
+          tc_fence_before_sync();
+          mbar_arrive(&mi.p_full[b]);
+        }
+        // ---- epilogue: normalise, stage bf16 rows in the (now idle) Q buffer, TMA store
+        mbar_wait(&mi.o_full[b], full_par(wt.o[b]), abort_flag, prm.status, W_OFULL);
+        ++wt.o[b];
+        tc_fence_after_sync();
+        const float inv_l = 1.0f / l_run;
+#pragma unroll
+        for (int q = 0; q < D / 32; ++q) {
+          uint32_t o[32];
+          tmem_ld32(tO + q * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int g4 = 0; g4 < 4; ++g4) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              pk[e] = pack_bf16x2(__uint_as_float(o[g4 * 8 + 2 * e]) * inv_l, __uint_as_float(o[g4 * 8 + 2 * e + 1]) * inv_l);
+            const int col = q * 32 + g4 * 8;
+            *reinterpret_cast<uint4*>(sQ[b] + (col / 64) * 16384 + sw128_offset(r, (col % 64) / 8)) =
+                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+        tc_fence_before_sync();
+        mbar_arrive(&mi.acc_free[b]);
+        const float lse2 = m_used + log2f(l_run);
+        if (token < prm.L) {
+          if (prm.lse) prm.lse[((size_t)c * prm.Hq + h) * prm.L + token] = lse2 * 0.6931471805599453f;
+          const int wi = token - (prm.L - prm.w);
+          if (wi >= 0) {
+            prm.win_lse[((size_t)c * prm.Hq + h) * prm.w + wi] = lse2 * 0.6931471805599453f;
+            if (within == 0) mi.lse2[(h - hkv * sch.G) * prm.w + wi] = lse2;   // G * w <= 256 entries per pass set
+          }
+        }
+        fence_proxy_async_smem();
+        named_barrier_sync(1 + b, 128);
+        if (r == 0) {
+          for (int a = 0; a < C::ATOMS; ++a) tma_store_4d(&tm_o, sQ[b] + a * 16384, a * 64, h, t * TILE, c);
+          tma_store_commit();
+          tma_store_wait_read();
+          mbar_arrive(&mi.q_free[b]);
+        }
+      }
+      if (within == 0) {
+        // ---- score sweep: this thread owns key (j * 128 + r); columns are the window rows
+        named_barrier_sync(3, 256);                           // lse2 complete and visible to both groups
+        for (int u = 0; u < n_pass; ++u) {
+          const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
+          const int rows_total = heads * prm.w;
+          const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
+          if (rows_b > 0) {
+            mbar_wait(&mi.q_full[b], full_par(wt.q[b]), abort_flag, prm.status, W_QFULL);
+            ++wt.q[b];
+            if (r < rows_b) rope_row_smem<D>(sQ[b], r, prm.rope_tab + (size_t)(prm.L - prm.w + (r % prm.w)) * (D / 2));
+            fence_proxy_async_smem();
+            mbar_arrive(&mi.q_rot[b]);
+          }
+          const float* lse_rows = mi.lse2 + u * Gs * prm.w + b * TILE;   // log-sum-exp of the window row on column n
+          for (int j = 0; j < sch.T; ++j) {
+            const int e = j & 1;
+            mbar_wait(&mi.t_full[e], full_par(wt.t[e]), abort_flag, prm.status, W_TFULL);
+            ++wt.t[e];
+            tc_fence_after_sync();
+            const int key = j * TILE + r;
+            const bool need_mask = (j * TILE + TILE - 1) > (prm.L - prm.w);
+            float part = 0.0f;
+            const uint32_t tT = tmem + e * 256 + b * 128 + lane_sel;
+            for (int c0 = 0; c0 < rows_b; c0 += 32) {
+              uint32_t sv[32];
+              tmem_ld32(tT + c0, sv);
+              tmem_wait_ld();
+#pragma unroll
+              for (int jj = 0; jj < 32; ++jj) {
+                const int ncol = c0 + jj;
+                if (ncol < rows_b) {
+                  float pv = fast_exp2(fmaf(__uint_as_float(sv[jj]), scale_log2, -lse_rows[ncol]));
+                  if (need_mask && key > prm.L - prm.w + ((b * TILE + ncol) % prm.w)) pv = 0.0f;
+                  part += pv;
+                }
+              }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&mi.t_free[e]);
+            if (b == 1) mi.xch[e][r] = part;
+            named_barrier_sync(3, 256);
+            if (b == 0 && key < prm.L) {
+              float* dst = prm.win_score + ((size_t)c * prm.Hkv + hkv) * prm.L + key;
+              const float total = part + mi.xch[e][r];
+              *dst = (u == 0) ? total : (*dst + total);
+            }
+          }
+          if (rows_b > 0) {
+            named_barrier_sync(1 + b, 128);                   // every thread of the group is past its last use of sQ[b]
+            if (r == 0) mbar_arrive(&mi.q_free[b]);
+          }
+        }
+      }
+    }
+    if (r == 0) tma_store_wait_all();
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == WARP_MMA) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ====================================================================================
+//                                   host launchers
+// ====================================================================================
+template <int D>
+static cudaError_t launch_prefill_t(const CUtensorMap* maps, const PrefillParams& prm, int grid, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Cfg<D>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  prefill_attn_kernel<D><<<grid, NUM_THREADS, Cfg<D>::SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_attn(const CUtensorMap* maps, const PrefillParams& prm, int d, int grid, cudaStream_t st) {
+  return d == 128 ? launch_prefill_t<128>(maps, prm, grid, st) : launch_prefill_t<64>(maps, prm, grid, st);
+}
+
+}  // namespace pc

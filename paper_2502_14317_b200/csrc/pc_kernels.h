@@ -1,0 +1,25 @@
+// Internal launcher declarations shared by the translation units of libpc.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstddef>
+#include <cstdint>
+
+namespace pc {
+
+// ---- pc_rope.cu
+// cos/sin table: tab[p * (d/2) + t] = (cos, sin)(  (pos0 + p) * theta^(-2t/d) ), fp64.
+void launch_rope_table(double2* tab, int n_pos, int d, double theta, int pos0, cudaStream_t st);
+// k_rot[c,p,h,:] = bf16( RoPE(k[c,p,h,:], position p) ), rotation evaluated in fp64.
+void launch_rope_keys(const void* k, const long long k_stride[3], void* k_rot, const double2* tab, int C, int L,
+                      int Hkv, int d, cudaStream_t st);
+
+// ---- pc_select_gather.cu
+void launch_chunk_score(const float* win_lse, int C, int n_per_chunk, float* score, cudaStream_t st);
+void launch_select_chunks(const float* score, int C, int m, int lower_is_better, int* kept, cudaStream_t st);
+cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
+                                 int* idx, cudaStream_t st);
+cudaError_t launch_gather_kv(const void* k_src, const void* v_src, const long long stride_elems[3], const int* kept,
+                             const int* idx, int m, int Hkv, int k, int d, void* k_out, void* v_out, int* pos_out,
+                             int sm_count, cudaStream_t st);
+
+}  // namespace pc

@@ -1,0 +1,103 @@
+"""GPU parity: pc_chunk_prefill_attn against the CPU oracle, element by element (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+import pc_inputs
+from oracle import parallelcomp_oracle as orc
+from tests.gpu_util import to_dev, to_bits, to_f64, check_attention_output, check_scores
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_and_compare(q, k, v, w, theta, want_lse=True):
+    import paper_2502_14317_b200 as pc
+    C, L, Hq, d = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    res = pc.chunk_prefill_attn(to_dev(q), to_dev(k), to_dev(v), w=w, rope_theta=theta, want_lse=want_lse)
+    torch.cuda.synchronize()
+    assert int(res["status"].item()) == 0, f"device wait ran out, code {int(res['status'].item())}"
+    O, LSE, k_rot = orc.local_attention(q, k, v, theta)
+    scale = 1.0 / np.sqrt(d)
+    S, O_win, LSE_win = orc.window_scores(orc.rope_bf16(q, theta), k_rot, v, w, scale)
+    # rotated keys: the rotation is evaluated in fp64 on both sides -> same bits
+    assert np.array_equal(to_bits(res["k_rot"]), k_rot), "k_rot differs from the oracle"
+    check_attention_output(to_f64(res["o"]), O)
+    lse = res["lse"].cpu().numpy().astype(np.float64)
+    assert np.abs(lse - LSE).max() <= 2e-3, f"LSE max err {np.abs(lse - LSE).max():.3e}"
+    win_lse = res["win_lse"].cpu().numpy().astype(np.float64)
+    assert np.abs(win_lse - LSE_win).max() <= 2e-3
+    got_S = res["win_score"].cpu().numpy()
+    check_scores(got_S, S, G, w, L)
+    assert np.allclose(got_S.sum(-1), G * w, rtol=1e-4)        # Eq. 6: G*w softmax rows, each summing to 1
+    return res
+
+
+def test_cfg0_full(cfg0_inputs):
+    cfg, inp = cfg0_inputs
+    _run_and_compare(inp["q"], inp["k"], inp["v"], cfg.w, cfg.rope_theta)
+
+
+@pytest.mark.parametrize("C,L,w,Hq,Hkv,d,theta", [
+    (2, 384, 64, 4, 1, 128, 500000.0),     # GQA G=4 (two head pairs), d=128, three query tiles
+    (2, 300, 16, 2, 2, 64, 10000.0),       # MHA (tile-pair mode), ragged last tile (300 = 2*128 + 44)
+    (1, 200, 128, 2, 1, 64, 10000.0),      # window spans two tiles, ragged
+    (3, 520, 8, 3, 3, 128, 10000.0),       # MHA, odd tile count (5 tiles), smallest window
+    (1, 100, 32, 8, 1, 64, 10000.0),       # single ragged tile, G*w = 256 window rows
+    (1, 640, 64, 8, 1, 128, 500000.0),     # G*w = 512 window rows: two score passes
+    (1, 130, 64, 1, 1, 64, 10000.0),       # single head, MHA, two tiles with a 2-token tail
+])
+def test_shapes(C, L, w, Hq, Hkv, d, theta):
+    rng = np.random.default_rng(L * 7 + Hq)
+    q = pc_inputs.f32_to_bf16_bits(rng.standard_normal((C, L, Hq, d)).astype(np.float32))
+    k = pc_inputs.f32_to_bf16_bits(rng.standard_normal((C, L, Hkv, d)).astype(np.float32))
+    v = pc_inputs.f32_to_bf16_bits(rng.standard_normal((C, L, Hkv, d)).astype(np.float32))
+    k[:, 0] = pc_inputs.f32_to_bf16_bits(pc_inputs.bf16_bits_to_f32(k[:, 0]) * np.float32(4.0))
+    _run_and_compare(q, k, v, w, theta)
+
+
+def test_deterministic_and_strided(cfg0_inputs):
+    import paper_2502_14317_b200 as pc
+    cfg, inp = cfg0_inputs
+    q, k, v = to_dev(inp["q"]), to_dev(inp["k"]), to_dev(inp["v"])
+    a = pc.chunk_prefill_attn(q, k, v, w=cfg.w, rope_theta=cfg.rope_theta)
+    b = pc.chunk_prefill_attn(q, k, v, w=cfg.w, rope_theta=cfg.rope_theta)
+    # head-major storage viewed token-major: same numbers through explicit strides
+    qh = q.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    kh = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    vh = v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    c = pc.chunk_prefill_attn(qh, kh, vh, w=cfg.w, rope_theta=cfg.rope_theta)
+    torch.cuda.synchronize()
+    for key in ("o", "k_rot", "win_score", "win_lse"):
+        assert torch.equal(a[key], b[key]), f"{key} not reproducible run to run"
+        assert torch.equal(a[key], c[key]), f"{key} differs for strided inputs"
+
+
+def test_argument_errors():
+    import paper_2502_14317_b200 as pc
+    q = torch.zeros((1, 256, 4, 64), dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros((1, 256, 2, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(pc.PcError, match="unsupported"):
+        pc.chunk_prefill_attn(q, k, k, w=24, rope_theta=1e4)           # window not a power of two
+    with pytest.raises(pc.PcError, match="invalid"):
+        pc.chunk_prefill_attn(q, k, k, w=256, rope_theta=1e4)          # window >= L
+    q96 = torch.zeros((1, 256, 4, 96), dtype=torch.bfloat16, device="cuda")
+    k96 = torch.zeros((1, 256, 2, 96), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(pc.PcError, match="unsupported"):
+        pc.chunk_prefill_attn(q96, k96, k96, w=16, rope_theta=1e4)     # head size
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    lib = pc.load_library()
+    import ctypes
+    from paper_2502_14317_b200.binding import _make_desc, _ptr
+    o = torch.empty_like(q)
+    desc = _make_desc(q, k, k, o, 16, 1e4, 0.0)
+    ws = torch.empty(64, dtype=torch.uint8, device="cuda")
+    S = torch.empty((1, 2, 256), dtype=torch.float32, device="cuda")
+    Lw = torch.empty((1, 4, 16), dtype=torch.float32, device="cuda")
+    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(k), _ptr(o), None, None, _ptr(S), _ptr(Lw),
+                                   None, _ptr(ws), ws.numel(), None)
+    assert rc == -3                                                     # PC_ERR_WORKSPACE
+    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), None, _ptr(k), _ptr(k), _ptr(o), None, None, _ptr(S), _ptr(Lw),
+                                   None, _ptr(ws), ws.numel(), None)
+    assert rc == -1                                                     # PC_ERR_INVALID_ARG
