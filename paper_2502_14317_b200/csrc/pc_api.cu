@@ -204,10 +204,123 @@ int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t* kv_str
 
 }  // extern "C"
 
-// ------------------------------------------------------------------------------------ parallel attention (placeholder until pc_parallel.cu lands)
-extern "C" {
-size_t pc_parallel_attn_workspace_bytes(int32_t, int32_t, int32_t, int32_t, int32_t, int32_t) { return 0; }
-int32_t pc_parallel_attn(int32_t, int32_t, int32_t, int32_t, int32_t, int32_t, const void*, int32_t, float, float,
-                         const void*, const void*, const void*, const void*, void*, float*, int32_t*, void*, size_t,
-                         void*) { return PC_ERR_UNSUPPORTED; }
+// ------------------------------------------------------------------------------------ parallel attention
+namespace {
+
+struct ParallelPlan {
+  int Gs, n_rg, n_cache_tiles, n_split, tiles_per_split;
+  size_t off_counter, off_table, off_ml, off_o, total;
+};
+
+// Split the keys so that the persistent grid has a few items per SM; every split keeps at
+// least two cache tiles.  The plan depends only on the sizes and the SM count.
+ParallelPlan parallel_plan(int B, int w, int Hq, int Hkv, int d, int Nk, int sm_count) {
+  ParallelPlan p;
+  const int G = Hq / Hkv;
+  p.Gs = (256 / w) < G ? (256 / w) : G;
+  p.n_rg = (G + p.Gs - 1) / p.Gs;
+  p.n_cache_tiles = (Nk + 127) / 128;
+  const long long base = (long long)B * Hkv * p.n_rg;
+  long long want = (4LL * sm_count + base - 1) / base;
+  long long cap = p.n_cache_tiles / 2;
+  if (cap < 1) cap = 1;
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  p.tiles_per_split = (int)((p.n_cache_tiles + want - 1) / want);
+  if (p.tiles_per_split < 1) p.tiles_per_split = 1;
+  p.n_split = p.n_cache_tiles > 0 ? (p.n_cache_tiles + p.tiles_per_split - 1) / p.tiles_per_split : 1;
+  size_t off = 0;
+  p.off_counter = off; off += ALIGN;
+  p.off_table = off; off += align_up((size_t)w * (d / 2) * sizeof(double2));
+  p.off_ml = off;
+  if (p.n_split > 1) off += align_up((size_t)B * Hq * p.n_split * w * 2 * sizeof(float));
+  p.off_o = off;
+  if (p.n_split > 1) off += align_up((size_t)B * Hq * p.n_split * w * d * sizeof(float));
+  p.total = off;
+  return p;
 }
+
+int32_t check_parallel_args(int B, int w, int Hq, int Hkv, int d, int Nk) {
+  if (B < 1 || w < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || Nk < 1) return PC_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
+  if (!pow2_between(w, 8, 128)) return PC_ERR_UNSUPPORTED;
+  if ((long long)B * Hq > (1 << 24) || Nk > (1 << 28)) return PC_ERR_UNSUPPORTED;
+  return PC_OK;
+}
+
+int plan_sm_count() {
+  const DeviceInfo& dev = device_info();
+  return dev.ok == 1 && dev.sm_count > 0 ? dev.sm_count : 148;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t pc_parallel_attn_workspace_bytes(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk) {
+  if (check_parallel_args(B, w, Hq, Hkv, d, Nk) != PC_OK) return 0;
+  return parallel_plan(B, w, Hq, Hkv, d, Nk, plan_sm_count()).total;
+}
+
+int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk, const void* q_win,
+                         int32_t q_pos0, float rope_theta, float softmax_scale, const void* k_cache,
+                         const void* v_cache, const void* k_win, const void* v_win, void* out, float* lse_out,
+                         int32_t* status_word, void* workspace, size_t workspace_bytes, void* stream) {
+  int32_t rc = check_parallel_args(B, w, Hq, Hkv, d, Nk);
+  if (rc != PC_OK) return rc;
+  if (!q_win || !k_cache || !v_cache || !k_win || !v_win || !out) return PC_ERR_INVALID_ARG;
+  if (!aligned16(q_win) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_win) || !aligned16(v_win) ||
+      !aligned16(out) || !aligned16(workspace))
+    return PC_ERR_INVALID_ARG;
+  if (q_pos0 < 0 || !(rope_theta > 0.0f) || softmax_scale < 0.0f) return PC_ERR_INVALID_ARG;
+  const DeviceInfo& dev = device_info();
+  if (dev.ok != 1) return PC_ERR_UNSUPPORTED;
+  const ParallelPlan plan = parallel_plan(B, w, Hq, Hkv, d, Nk, dev.sm_count);
+  if (!workspace || workspace_bytes < plan.total) return PC_ERR_WORKSPACE;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  int* counter = reinterpret_cast<int*>(ws + plan.off_counter);
+  double2* table = reinterpret_cast<double2*>(ws + plan.off_table);
+
+  CUtensorMap maps[5];
+  const uint64_t ud = (uint64_t)d;
+  const uint64_t qw_dims[4] = {ud, (uint64_t)Hq, (uint64_t)w, (uint64_t)B};
+  const uint64_t qw_str[3] = {ud, (uint64_t)Hq * ud, (uint64_t)w * Hq * ud};
+  const uint64_t kc_dims[4] = {ud, (uint64_t)Nk, (uint64_t)Hkv, (uint64_t)B};
+  const uint64_t kc_str[3] = {ud, (uint64_t)Nk * ud, (uint64_t)Hkv * Nk * ud};
+  const uint64_t kw_dims[4] = {ud, (uint64_t)Hkv, (uint64_t)w, (uint64_t)B};
+  const uint64_t kw_str[3] = {ud, (uint64_t)Hkv * ud, (uint64_t)w * Hkv * ud};
+  const uint32_t box_qw[4] = {64, 1, (uint32_t)w, 1};
+  const uint32_t box_kc[4] = {64, 128, 1, 1};
+  const uint32_t box_kw[4] = {64, 1, 128, 1};
+  if (!pc::make_tmap_bf16_4d(&maps[0], q_win, qw_dims, qw_str, box_qw) ||
+      !pc::make_tmap_bf16_4d(&maps[1], k_cache, kc_dims, kc_str, box_kc) ||
+      !pc::make_tmap_bf16_4d(&maps[2], v_cache, kc_dims, kc_str, box_kc) ||
+      !pc::make_tmap_bf16_4d(&maps[3], k_win, kw_dims, kw_str, box_kw) ||
+      !pc::make_tmap_bf16_4d(&maps[4], v_win, kw_dims, kw_str, box_kw))
+    return PC_ERR_CUDA;
+
+  if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return PC_ERR_CUDA;
+  pc::launch_rope_table(table, w, d, (double)rope_theta, q_pos0, st);
+
+  pc::ParallelParams prm;
+  prm.B = B; prm.w = w; prm.Hq = Hq; prm.Hkv = Hkv; prm.Nk = Nk;
+  prm.Gs = plan.Gs; prm.n_rg = plan.n_rg;
+  prm.n_cache_tiles = plan.n_cache_tiles; prm.n_split = plan.n_split; prm.tiles_per_split = plan.tiles_per_split;
+  const double scale = softmax_scale > 0.0f ? (double)softmax_scale : 1.0 / std::sqrt((double)d);
+  prm.scale_log2 = (float)(scale * 1.4426950408889634);
+  prm.rope_tab = table;
+  prm.part_ml = reinterpret_cast<float*>(ws + plan.off_ml);
+  prm.part_o = reinterpret_cast<float*>(ws + plan.off_o);
+  prm.out = static_cast<__nv_bfloat16*>(out);
+  prm.lse_out = lse_out;
+  prm.status = status_word;
+  prm.counter = counter;
+  const long long n_items = (long long)B * Hkv * plan.n_rg * plan.n_split;
+  const int grid = (int)(n_items < dev.sm_count ? n_items : dev.sm_count);
+  if (pc::launch_parallel_attn(maps, prm, d, grid, st) != cudaSuccess) return PC_ERR_CUDA;
+  return PC_OK;
+}
+
+}  // extern "C"

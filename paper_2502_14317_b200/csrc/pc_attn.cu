@@ -244,6 +244,146 @@ struct Waits {                                 // how many times each barrier ha
 __device__ __forceinline__ uint32_t full_par(uint32_t n) { return n & 1u; }          // n-th use of a "full" barrier
 __device__ __forceinline__ uint32_t free_par(uint32_t n) { return (n & 1u) ^ 1u; }   // before the n-th use of a resource
 
+// ------------------------------------------------------------------ shared pieces of the three roles
+struct Ctx {
+  Misc* mi;
+  uint8_t* sQ[2];
+  uint8_t* ring;
+  uint32_t tmem;
+  volatile int* abort_flag;
+  int* status;
+};
+
+__device__ __forceinline__ void init_barriers(Misc& mi) {
+  for (int b = 0; b < 2; ++b) {
+    mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 128); mbar_init(&mi.q_free[b], 1);
+    mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_full[b], 128); mbar_init(&mi.o_full[b], 1);
+    mbar_init(&mi.acc_free[b], 128);
+    mbar_init(&mi.item_full[b], 1); mbar_init(&mi.item_empty[b], 257);
+    mbar_init(&mi.t_full[b], 1); mbar_init(&mi.t_free[b], 256);
+  }
+  for (int s = 0; s < NS; ++s) { mbar_init(&mi.kv_full[s], 1); mbar_init(&mi.kv_free[s], 1); }
+  mi.abort_flag = 0;
+  fence_mbar_init();
+}
+
+// producer: publish the next work item (dynamic queue); returns it
+__device__ __forceinline__ int producer_next_item(const Ctx& cx, Waits& wt, int* counter, int n_items) {
+  Misc& mi = *cx.mi;
+  const int slot = wt.item & 1;
+  mbar_wait(&mi.item_empty[slot], free_par(wt.item >> 1), cx.abort_flag, cx.status, W_ITEM);
+  int item = atomicAdd(counter, 1);
+  if (item >= n_items || *cx.abort_flag) item = ITEM_DONE;
+  mi.item_slot[slot] = item;
+  mbar_arrive(&mi.item_full[slot]);
+  ++wt.item;
+  return item;
+}
+// consumers: read the next work item
+__device__ __forceinline__ int consumer_next_item(const Ctx& cx, Waits& wt) {
+  Misc& mi = *cx.mi;
+  const int slot = wt.item & 1;
+  mbar_wait(&mi.item_full[slot], full_par(wt.item >> 1), cx.abort_flag, cx.status, W_ITEM);
+  const int item = mi.item_slot[slot];
+  mbar_arrive(&mi.item_empty[slot]);
+  ++wt.item;
+  return item;
+}
+
+// producer: one 128 x D tile into the next ring stage; (c1, c2, c3) are the outer TMA coordinates
+template <int D>
+__device__ __forceinline__ void producer_ring_tile(const Ctx& cx, Waits& wt, const CUtensorMap* tmap, int c1, int c2,
+                                                   int c3) {
+  using C = Cfg<D>;
+  Misc& mi = *cx.mi;
+  const int st = wt.kv % NS;
+  mbar_wait(&mi.kv_free[st], free_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFREE);
+  mbar_arrive_expect_tx(&mi.kv_full[st], C::TILE_BYTES);
+  for (int a = 0; a < C::ATOMS; ++a)
+    tma_load_4d(cx.ring + st * C::TILE_BYTES + a * 16384, tmap, &mi.kv_full[st], a * 64, c1, c2, c3);
+  ++wt.kv;
+}
+
+// producer: before exit, every copy it issued must have landed
+__device__ __forceinline__ void producer_drain(const Ctx& cx, const Waits& wt) {
+  Misc& mi = *cx.mi;
+  for (uint32_t i = (wt.kv > NS ? wt.kv - NS : 0); i < wt.kv; ++i) mbar_wait_drain(&mi.kv_full[i % NS], full_par(i / NS));
+  for (int b = 0; b < 2; ++b)
+    if (wt.q[b] > 0) mbar_wait_drain(&mi.q_full[b], full_par(wt.q[b] - 1));
+}
+
+// issuer: the flash loop for a pair of query blocks sharing K/V tiles.  Ring order is
+// K0, V0, K1, V1, ...; block b takes part in its first nb[b] tiles.
+template <int D>
+__device__ __forceinline__ void mma_flash_pair(const Ctx& cx, Waits& wt, const bool has[2], const int nb[2]) {
+  using C = Cfg<D>;
+  Misc& mi = *cx.mi;
+  const uint32_t ring_u32 = smem_u32(cx.ring);
+  const uint32_t q_u32[2] = {smem_u32(cx.sQ[0]), smem_u32(cx.sQ[1])};
+  const uint32_t tS[2] = {cx.tmem + 0, cx.tmem + 128}, tO[2] = {cx.tmem + 256, cx.tmem + 384};
+  const int n = nb[1] > nb[0] ? nb[1] : nb[0];
+  // accumulators and score buffers of earlier work must have been read out
+  for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
+  for (int e = 0; e < 2; ++e) mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
+  for (int b = 0; b < 2; ++b)
+    if (has[b]) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
+  tc_fence_after_sync();
+  {  // S(0)
+    const int st = wt.kv % NS;
+    mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
+    tc_fence_after_sync();
+    for (int b = 0; b < 2; ++b)
+      if (has[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
+    mma_commit(&mi.kv_free[st]);
+    ++wt.kv;
+  }
+  for (int j = 0; j < n; ++j) {
+    const int st_v = wt.kv % NS;
+    mbar_wait(&mi.kv_full[st_v], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
+    ++wt.kv;
+    int st_k = 0;
+    const bool more = j + 1 < n;
+    if (more) {
+      st_k = wt.kv % NS;
+      mbar_wait(&mi.kv_full[st_k], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
+      ++wt.kv;
+    }
+    for (int b = 0; b < 2; ++b) {
+      if (!has[b] || j >= nb[b]) continue;
+      mbar_wait(&mi.p_full[b], full_par(wt.p[b]), cx.abort_flag, cx.status, W_PFULL);
+      ++wt.p[b];
+      tc_fence_after_sync();
+      issue_pv<D>(tO[b], tS[b], ring_u32 + st_v * C::TILE_BYTES, j > 0);
+      if (j == nb[b] - 1) mma_commit(&mi.o_full[b]);
+      if (j + 1 < nb[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st_k * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
+    }
+    mma_commit(&mi.kv_free[st_v]);
+    if (more) mma_commit(&mi.kv_free[st_k]);
+  }
+  for (int b = 0; b < 2; ++b) if (has[b]) ++wt.acc[b];
+}
+
+// softmax group: online softmax over n key tiles for this thread's row; vis(j) = visible
+// columns of tile j.  Leaves (m_used, l_run); the accumulator O_b stays in TMEM.
+template <int D, class VisFn>
+__device__ __forceinline__ void wg_flash_loop(const Ctx& cx, Waits& wt, int b, uint32_t tS, uint32_t tO, int n,
+                                              float scale_log2, VisFn vis, float& m_used, float& l_run) {
+  Misc& mi = *cx.mi;
+  m_used = -INFINITY;
+  l_run = 0.0f;
+  for (int j = 0; j < n; ++j) {
+    mbar_wait(&mi.s_full[b], full_par(wt.s[b]), cx.abort_flag, cx.status, W_SFULL);
+    ++wt.s[b];
+    tc_fence_after_sync();
+    softmax_tile<D>(tS, tO, vis(j), j == 0, scale_log2, m_used, l_run);
+    tc_fence_before_sync();
+    mbar_arrive(&mi.p_full[b]);
+  }
+  mbar_wait(&mi.o_full[b], full_par(wt.o[b]), cx.abort_flag, cx.status, W_OFULL);
+  ++wt.o[b];
+  tc_fence_after_sync();
+}
+
 }  // namespace
 
 // ====================================================================================
@@ -258,34 +398,26 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   Misc& mi = *reinterpret_cast<Misc*>(smem + C::OFF_MISC);
-  uint8_t* sQ[2] = {smem + C::OFF_Q, smem + C::OFF_Q + C::TILE_BYTES};
-  uint8_t* ring = smem + C::OFF_RING;
-  volatile int* abort_flag = &mi.abort_flag;
+  Ctx cx;
+  cx.mi = &mi;
+  cx.sQ[0] = smem + C::OFF_Q;
+  cx.sQ[1] = smem + C::OFF_Q + C::TILE_BYTES;
+  cx.ring = smem + C::OFF_RING;
+  cx.abort_flag = &mi.abort_flag;
+  cx.status = prm.status;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Sched sch = make_sched(prm);
-  const int n_groups = prm.C * prm.Hkv;
-  const int n_items = n_groups * sch.ipg;
+  const int n_items = prm.C * prm.Hkv * sch.ipg;
   const int Gs = (256 / prm.w) < sch.G ? (256 / prm.w) : sch.G;      // q-heads per score pass
   const int n_pass = (sch.G + Gs - 1) / Gs;
 
-  if (tid == 0) {
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 128); mbar_init(&mi.q_free[b], 1);
-      mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_full[b], 128); mbar_init(&mi.o_full[b], 1);
-      mbar_init(&mi.acc_free[b], 128);
-      mbar_init(&mi.item_full[b], 1); mbar_init(&mi.item_empty[b], 257);
-      mbar_init(&mi.t_full[b], 1); mbar_init(&mi.t_free[b], 256);
-    }
-    for (int s = 0; s < NS; ++s) { mbar_init(&mi.kv_full[s], 1); mbar_init(&mi.kv_free[s], 1); }
-    mi.abort_flag = 0;
-    fence_mbar_init();
-  }
+  if (tid == 0) init_barriers(mi);
   if (warp == WARP_MMA) tmem_alloc(&mi.tmem_base, 512);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem = mi.tmem_base;
+  cx.tmem = mi.tmem_base;
 
   Waits wt;
 
@@ -294,14 +426,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_qw);
       while (true) {
-        // ---- fetch and publish the next item
-        const int slot = wt.item & 1;
-        mbar_wait(&mi.item_empty[slot], free_par(wt.item >> 1), abort_flag, prm.status, W_ITEM);
-        int item = atomicAdd(prm.counter, 1);
-        if (item >= n_items || *abort_flag) item = ITEM_DONE;
-        mi.item_slot[slot] = item;
-        mbar_arrive(&mi.item_full[slot]);
-        ++wt.item;
+        const int item = producer_next_item(cx, wt, prm.counter, n_items);
         if (item == ITEM_DONE) break;
         const int group = item / sch.ipg, within = item % sch.ipg;
         const int c = group / prm.Hkv, hkv = group % prm.Hkv;
@@ -311,22 +436,16 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int b = 0; b < 2; ++b) {
             const int h = b ? it.hB : it.hA, t = b ? it.tB : it.tA;
             if (h < 0) continue;
-            mbar_wait(&mi.q_free[b], free_par(wt.q[b]), abort_flag, prm.status, W_QFREE);
+            mbar_wait(&mi.q_free[b], free_par(wt.q[b]), cx.abort_flag, cx.status, W_QFREE);
             mbar_arrive_expect_tx(&mi.q_full[b], C::TILE_BYTES);
-            for (int a = 0; a < C::ATOMS; ++a) tma_load_4d(sQ[b] + a * 16384, &tm_q, &mi.q_full[b], a * 64, h, t * TILE, c);
+            for (int a = 0; a < C::ATOMS; ++a)
+              tma_load_4d(cx.sQ[b] + a * 16384, &tm_q, &mi.q_full[b], a * 64, h, t * TILE, c);
             ++wt.q[b];
           }
           const int n = (it.hB >= 0 ? it.tB : it.tA) + 1;
           for (int j = 0; j < n; ++j) {
-            for (int kv = 0; kv < 2; ++kv) {                       // K_j then V_j
-              const int st = wt.kv % NS;
-              mbar_wait(&mi.kv_free[st], free_par(wt.kv / NS), abort_flag, prm.status, W_KVFREE);
-              mbar_arrive_expect_tx(&mi.kv_full[st], C::TILE_BYTES);
-              for (int a = 0; a < C::ATOMS; ++a)
-                tma_load_4d(ring + st * C::TILE_BYTES + a * 16384, kv ? &tm_v : &tm_k, &mi.kv_full[st], a * 64, hkv,
-                            j * TILE, c);
-              ++wt.kv;
-            }
+            producer_ring_tile<D>(cx, wt, &tm_k, hkv, j * TILE, c);
+            producer_ring_tile<D>(cx, wt, &tm_v, hkv, j * TILE, c);
           }
         }
         if (within == 0) {
@@ -337,45 +456,30 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int b = 0; b < 2; ++b) {
               const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
               if (rows_b == 0) continue;
-              mbar_wait(&mi.q_free[b], free_par(wt.q[b]), abort_flag, prm.status, W_QFREE);
+              mbar_wait(&mi.q_free[b], free_par(wt.q[b]), cx.abort_flag, cx.status, W_QFREE);
               mbar_arrive_expect_tx(&mi.q_full[b], rows_b * D * 2);
               for (int r0 = 0; r0 < rows_b; r0 += prm.w) {
                 const int g = u * Gs + (b * TILE + r0) / prm.w;
                 for (int a = 0; a < C::ATOMS; ++a)
-                  tma_load_4d(sQ[b] + a * 16384 + r0 * 128, &tm_qw, &mi.q_full[b], a * 64, hkv * sch.G + g,
+                  tma_load_4d(cx.sQ[b] + a * 16384 + r0 * 128, &tm_qw, &mi.q_full[b], a * 64, hkv * sch.G + g,
                               prm.L - prm.w, c);
               }
               ++wt.q[b];
             }
-            for (int j = 0; j < sch.T; ++j) {
-              const int st = wt.kv % NS;
-              mbar_wait(&mi.kv_free[st], free_par(wt.kv / NS), abort_flag, prm.status, W_KVFREE);
-              mbar_arrive_expect_tx(&mi.kv_full[st], C::TILE_BYTES);
-              for (int a = 0; a < C::ATOMS; ++a)
-                tma_load_4d(ring + st * C::TILE_BYTES + a * 16384, &tm_k, &mi.kv_full[st], a * 64, hkv, j * TILE, c);
-              ++wt.kv;
-            }
+            for (int j = 0; j < sch.T; ++j) producer_ring_tile<D>(cx, wt, &tm_k, hkv, j * TILE, c);
           }
         }
       }
-      // drain: every copy this thread issued must have landed before the CTA exits
-      for (uint32_t i = (wt.kv > NS ? wt.kv - NS : 0); i < wt.kv; ++i) mbar_wait_drain(&mi.kv_full[i % NS], full_par(i / NS));
-      for (int b = 0; b < 2; ++b)
-        if (wt.q[b] > 0) mbar_wait_drain(&mi.q_full[b], full_par(wt.q[b] - 1));
+      producer_drain(cx, wt);
     }
     __syncwarp();
   } else if (warp == WARP_MMA) {
     // ================================================================ tcgen05 issuer
     if (lane == 0) {
-      const uint32_t ring_u32 = smem_u32(ring);
-      const uint32_t q_u32[2] = {smem_u32(sQ[0]), smem_u32(sQ[1])};
-      const uint32_t tS[2] = {tmem + 0, tmem + 128}, tO[2] = {tmem + 256, tmem + 384};
+      const uint32_t ring_u32 = smem_u32(cx.ring);
+      const uint32_t q_u32[2] = {smem_u32(cx.sQ[0]), smem_u32(cx.sQ[1])};
       while (true) {
-        const int slot = wt.item & 1;
-        mbar_wait(&mi.item_full[slot], full_par(wt.item >> 1), abort_flag, prm.status, W_ITEM);
-        const int item = mi.item_slot[slot];
-        mbar_arrive(&mi.item_empty[slot]);
-        ++wt.item;
+        const int item = consumer_next_item(cx, wt);
         if (item == ITEM_DONE) break;
         const int group = item / sch.ipg, within = item % sch.ipg;
         const int hkv = group % prm.Hkv;
@@ -384,66 +488,26 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const SubItem it = decode_sub(sch, hkv, within, sub);
           const bool has[2] = {true, it.hB >= 0};
           const int nb[2] = {it.tA + 1, it.hB >= 0 ? it.tB + 1 : 0};
-          const int n = nb[1] > nb[0] ? nb[1] : nb[0];
-          // accumulators and score buffers of earlier work must have been read out
-          for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), abort_flag, prm.status, W_ACCFREE);
-          for (int e = 0; e < 2; ++e) mbar_wait(&mi.t_free[e], free_par(wt.t[e]), abort_flag, prm.status, W_TFREE);
-          for (int b = 0; b < 2; ++b)
-            if (has[b]) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), abort_flag, prm.status, W_QROT); ++wt.q[b]; }
-          tc_fence_after_sync();
-          // S(0)
-          {
-            const int st = wt.kv % NS;
-            mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), abort_flag, prm.status, W_KVFULL);
-            tc_fence_after_sync();
-            for (int b = 0; b < 2; ++b)
-              if (has[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
-            mma_commit(&mi.kv_free[st]);
-            ++wt.kv;
-          }
-          for (int j = 0; j < n; ++j) {
-            const int st_v = wt.kv % NS;
-            mbar_wait(&mi.kv_full[st_v], full_par(wt.kv / NS), abort_flag, prm.status, W_KVFULL);
-            ++wt.kv;
-            int st_k = 0;
-            const bool more = j + 1 < n;
-            if (more) {
-              st_k = wt.kv % NS;
-              mbar_wait(&mi.kv_full[st_k], full_par(wt.kv / NS), abort_flag, prm.status, W_KVFULL);
-              ++wt.kv;
-            }
-            for (int b = 0; b < 2; ++b) {
-              if (!has[b] || j >= nb[b]) continue;
-              mbar_wait(&mi.p_full[b], full_par(wt.p[b]), abort_flag, prm.status, W_PFULL);
-              ++wt.p[b];
-              tc_fence_after_sync();
-              issue_pv<D>(tO[b], tS[b], ring_u32 + st_v * C::TILE_BYTES, j > 0);
-              if (j == nb[b] - 1) mma_commit(&mi.o_full[b]);
-              if (j + 1 < nb[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st_k * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
-            }
-            mma_commit(&mi.kv_free[st_v]);
-            if (more) mma_commit(&mi.kv_free[st_k]);
-          }
-          for (int b = 0; b < 2; ++b) if (has[b]) ++wt.acc[b];
+          mma_flash_pair<D>(cx, wt, has, nb);
         }
         if (within == 0) {
-          for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), abort_flag, prm.status, W_ACCFREE);
+          for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
           for (int u = 0; u < n_pass; ++u) {
             const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
             const int rows_total = heads * prm.w;
             const int rows[2] = {rows_total < TILE ? rows_total : TILE, rows_total > TILE ? rows_total - TILE : 0};
             for (int b = 0; b < 2; ++b)
-              if (rows[b] > 0) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), abort_flag, prm.status, W_QROT); ++wt.q[b]; }
+              if (rows[b] > 0) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
             for (int j = 0; j < sch.T; ++j) {
               const int e = j & 1;
-              mbar_wait(&mi.t_free[e], free_par(wt.t[e]), abort_flag, prm.status, W_TFREE);
+              mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
               const int st = wt.kv % NS;
-              mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), abort_flag, prm.status, W_KVFULL);
+              mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
               ++wt.kv;
               tc_fence_after_sync();
               for (int b = 0; b < 2; ++b)
                 if (rows[b] > 0)
-                  issue_kq<D>(tmem + e * 256 + b * 128, ring_u32 + st * C::TILE_BYTES, q_u32[b], (rows[b] + 15) & ~15);
+                  issue_kq<D>(cx.tmem + e * 256 + b * 128, ring_u32 + st * C::TILE_BYTES, q_u32[b], (rows[b] + 15) & ~15);
               mma_commit(&mi.t_full[e]);
               mma_commit(&mi.kv_free[st]);
               ++wt.t[e];
@@ -458,14 +522,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int b = warp >> 2;                                 // block / group index
     const int r = tid & 127;                                 // row in the block = TMEM lane
     const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + b * 128 + lane_sel, tO = tmem + 256 + b * 128 + lane_sel;
+    const uint32_t tS = cx.tmem + b * 128 + lane_sel, tO = cx.tmem + 256 + b * 128 + lane_sel;
     const float scale_log2 = prm.scale_log2;
+    uint8_t* const myQ = cx.sQ[b];
     while (true) {
-      const int slot = wt.item & 1;
-      mbar_wait(&mi.item_full[slot], full_par(wt.item >> 1), abort_flag, prm.status, W_ITEM);
-      const int item = mi.item_slot[slot];
-      mbar_arrive(&mi.item_empty[slot]);
-      ++wt.item;
+      const int item = consumer_next_item(cx, wt);
       if (item == ITEM_DONE) break;
       const int group = item / sch.ipg, within = item % sch.ipg;
       const int c = group / prm.Hkv, hkv = group % prm.Hkv;
@@ -476,27 +537,17 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (h < 0) continue;
         const int token = t * TILE + r;
         // ---- Q prologue: rotate this thread's row in shared memory
-        mbar_wait(&mi.q_full[b], full_par(wt.q[b]), abort_flag, prm.status, W_QFULL);
+        mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QFULL);
         ++wt.q[b];
-        if (token < prm.L) rope_row_smem<D>(sQ[b], r, prm.rope_tab + (size_t)token * (D / 2));
+        if (token < prm.L) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)token * (D / 2));
         fence_proxy_async_smem();
         mbar_arrive(&mi.q_rot[b]);
-        // ---- main loop over key tiles
-        float m_used = -INFINITY, l_run = 0.0f;
+        // ---- main loop over key tiles (causal: keys <= token; only the diagonal tile is masked)
+        float m_used, l_run;
         const int n = t + 1;
-        for (int j = 0; j < n; ++j) {
-          mbar_wait(&mi.s_full[b], full_par(wt.s[b]), abort_flag, prm.status, W_SFULL);
-          ++wt.s[b];
-          tc_fence_after_sync();
-          const int vis = (j == n - 1) ? (token - j * TILE + 1) : TILE;      // causal: keys <= token
-          softmax_tile<D>(tS, tO, vis, j == 0, scale_log2, m_used, l_run);
-          tc_fence_before_sync();
-          mbar_arrive(&mi.p_full[b]);
-        }
+        wg_flash_loop<D>(cx, wt, b, tS, tO, n, scale_log2,
+                         [&](int j) { return (j == n - 1) ? (token - j * TILE + 1) : TILE; }, m_used, l_run);
         // ---- epilogue: normalise, stage bf16 rows in the (now idle) Q buffer, TMA store
-        mbar_wait(&mi.o_full[b], full_par(wt.o[b]), abort_flag, prm.status, W_OFULL);
-        ++wt.o[b];
-        tc_fence_after_sync();
         const float inv_l = 1.0f / l_run;
 #pragma unroll
         for (int q = 0; q < D / 32; ++q) {
@@ -510,7 +561,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int e = 0; e < 4; ++e)
               pk[e] = pack_bf16x2(__uint_as_float(o[g4 * 8 + 2 * e]) * inv_l, __uint_as_float(o[g4 * 8 + 2 * e + 1]) * inv_l);
             const int col = q * 32 + g4 * 8;
-            *reinterpret_cast<uint4*>(sQ[b] + (col / 64) * 16384 + sw128_offset(r, (col % 64) / 8)) =
+            *reinterpret_cast<uint4*>(myQ + (col / 64) * 16384 + sw128_offset(r, (col % 64) / 8)) =
                 make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
@@ -522,13 +573,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int wi = token - (prm.L - prm.w);
           if (wi >= 0) {
             prm.win_lse[((size_t)c * prm.Hq + h) * prm.w + wi] = lse2 * 0.6931471805599453f;
-            if (within == 0) mi.lse2[(h - hkv * sch.G) * prm.w + wi] = lse2;   // G * w <= 256 entries per pass set
+            if (within == 0) mi.lse2[(h - hkv * sch.G) * prm.w + wi] = lse2;
           }
         }
         fence_proxy_async_smem();
         named_barrier_sync(1 + b, 128);
         if (r == 0) {
-          for (int a = 0; a < C::ATOMS; ++a) tma_store_4d(&tm_o, sQ[b] + a * 16384, a * 64, h, t * TILE, c);
+          for (int a = 0; a < C::ATOMS; ++a) tma_store_4d(&tm_o, myQ + a * 16384, a * 64, h, t * TILE, c);
           tma_store_commit();
           tma_store_wait_read();
           mbar_arrive(&mi.q_free[b]);
@@ -542,22 +593,22 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int rows_total = heads * prm.w;
           const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
           if (rows_b > 0) {
-            mbar_wait(&mi.q_full[b], full_par(wt.q[b]), abort_flag, prm.status, W_QFULL);
+            mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QFULL);
             ++wt.q[b];
-            if (r < rows_b) rope_row_smem<D>(sQ[b], r, prm.rope_tab + (size_t)(prm.L - prm.w + (r % prm.w)) * (D / 2));
+            if (r < rows_b) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)(prm.L - prm.w + (r % prm.w)) * (D / 2));
             fence_proxy_async_smem();
             mbar_arrive(&mi.q_rot[b]);
           }
           const float* lse_rows = mi.lse2 + u * Gs * prm.w + b * TILE;   // log-sum-exp of the window row on column n
           for (int j = 0; j < sch.T; ++j) {
             const int e = j & 1;
-            mbar_wait(&mi.t_full[e], full_par(wt.t[e]), abort_flag, prm.status, W_TFULL);
+            mbar_wait(&mi.t_full[e], full_par(wt.t[e]), cx.abort_flag, cx.status, W_TFULL);
             ++wt.t[e];
             tc_fence_after_sync();
             const int key = j * TILE + r;
             const bool need_mask = (j * TILE + TILE - 1) > (prm.L - prm.w);
             float part = 0.0f;
-            const uint32_t tT = tmem + e * 256 + b * 128 + lane_sel;
+            const uint32_t tT = cx.tmem + e * 256 + b * 128 + lane_sel;
             for (int c0 = 0; c0 < rows_b; c0 += 32) {
               uint32_t sv[32];
               tmem_ld32(tT + c0, sv);
@@ -567,7 +618,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const int ncol = c0 + jj;
                 if (ncol < rows_b) {
                   float pv = fast_exp2(fmaf(__uint_as_float(sv[jj]), scale_log2, -lse_rows[ncol]));
-                  if (need_mask && key > prm.L - prm.w + ((b * TILE + ncol) % prm.w)) pv = 0.0f;
+                  if (need_mask && key > prm.L - prm.w + (ncol % prm.w)) pv = 0.0f;
                   part += pv;
                 }
               }
@@ -596,8 +647,222 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   if (warp == WARP_MMA) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(cx.tmem, 512);
   }
+}
+
+// ====================================================================================
+//                          PARALLEL (GLOBAL) ATTENTION KERNEL
+// ====================================================================================
+// Item = (sequence, kv-head, row group, key split).  The rows of an item are the w window
+// queries of up to 256/w q-heads of one kv-head, packed head-major into the two 128-row
+// blocks; both blocks stream the same cache tiles, and the last split appends the
+// window's own keys (causal inside the window).
+template <int D>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_constant__ CUtensorMap tm_kc,
+                     const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kw,
+                     const __grid_constant__ CUtensorMap tm_vw, const __grid_constant__ ParallelParams prm) {
+  using C = Cfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  Misc& mi = *reinterpret_cast<Misc*>(smem + C::OFF_MISC);
+  Ctx cx;
+  cx.mi = &mi;
+  cx.sQ[0] = smem + C::OFF_Q;
+  cx.sQ[1] = smem + C::OFF_Q + C::TILE_BYTES;
+  cx.ring = smem + C::OFF_RING;
+  cx.abort_flag = &mi.abort_flag;
+  cx.status = prm.status;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = prm.Hq / prm.Hkv;
+  const int n_items = prm.B * prm.Hkv * prm.n_rg * prm.n_split;
+
+  if (tid == 0) init_barriers(mi);
+  if (warp == WARP_MMA) tmem_alloc(&mi.tmem_base, 512);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  cx.tmem = mi.tmem_base;
+
+  Waits wt;
+
+  // item -> (seq, hkv, rg, split) and its tile range / row counts
+  struct Dec { int seq, hkv, g0, split, rows[2], j0, n_cache, n; };
+  auto decode = [&](int item) {
+    Dec d;
+    d.split = item % prm.n_split;
+    int x = item / prm.n_split;
+    const int rg = x % prm.n_rg; x /= prm.n_rg;
+    d.hkv = x % prm.Hkv;
+    d.seq = x / prm.Hkv;
+    d.g0 = rg * prm.Gs;
+    const int heads = (G - d.g0) < prm.Gs ? (G - d.g0) : prm.Gs;
+    const int rows_total = heads * prm.w;
+    d.rows[0] = rows_total < TILE ? rows_total : TILE;
+    d.rows[1] = rows_total > TILE ? rows_total - TILE : 0;
+    d.j0 = d.split * prm.tiles_per_split;
+    const int j1 = (d.j0 + prm.tiles_per_split) < prm.n_cache_tiles ? (d.j0 + prm.tiles_per_split) : prm.n_cache_tiles;
+    d.n_cache = j1 - d.j0;
+    d.n = d.n_cache + (d.split == prm.n_split - 1 ? 1 : 0);
+    return d;
+  };
+
+  if (warp == WARP_PRODUCER) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_qw); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
+      while (true) {
+        const int item = producer_next_item(cx, wt, prm.counter, n_items);
+        if (item == ITEM_DONE) break;
+        const Dec d = decode(item);
+        for (int b = 0; b < 2; ++b) {
+          if (d.rows[b] == 0) continue;
+          mbar_wait(&mi.q_free[b], free_par(wt.q[b]), cx.abort_flag, cx.status, W_QFREE);
+          mbar_arrive_expect_tx(&mi.q_full[b], d.rows[b] * D * 2);
+          for (int r0 = 0; r0 < d.rows[b]; r0 += prm.w) {
+            const int g = d.g0 + (b * TILE + r0) / prm.w;
+            for (int a = 0; a < C::ATOMS; ++a)
+              tma_load_4d(cx.sQ[b] + a * 16384 + r0 * 128, &tm_qw, &mi.q_full[b], a * 64, d.hkv * G + g, 0, d.seq);
+          }
+          ++wt.q[b];
+        }
+        for (int jj = 0; jj < d.n; ++jj) {
+          if (jj < d.n_cache) {
+            producer_ring_tile<D>(cx, wt, &tm_kc, (d.j0 + jj) * TILE, d.hkv, d.seq);
+            producer_ring_tile<D>(cx, wt, &tm_vc, (d.j0 + jj) * TILE, d.hkv, d.seq);
+          } else {
+            producer_ring_tile<D>(cx, wt, &tm_kw, d.hkv, 0, d.seq);
+            producer_ring_tile<D>(cx, wt, &tm_vw, d.hkv, 0, d.seq);
+          }
+        }
+      }
+      producer_drain(cx, wt);
+    }
+    __syncwarp();
+  } else if (warp == WARP_MMA) {
+    if (lane == 0) {
+      while (true) {
+        const int item = consumer_next_item(cx, wt);
+        if (item == ITEM_DONE) break;
+        const Dec d = decode(item);
+        const bool has[2] = {d.rows[0] > 0, d.rows[1] > 0};
+        const int nb[2] = {has[0] ? d.n : 0, has[1] ? d.n : 0};
+        mma_flash_pair<D>(cx, wt, has, nb);
+      }
+    }
+    __syncwarp();
+  } else {
+    const int b = warp >> 2;
+    const int r = tid & 127;
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t tS = cx.tmem + b * 128 + lane_sel, tO = cx.tmem + 256 + b * 128 + lane_sel;
+    uint8_t* const myQ = cx.sQ[b];
+    const int wi = r % prm.w;                                 // window index of this row (128 % w == 0)
+    while (true) {
+      const int item = consumer_next_item(cx, wt);
+      if (item == ITEM_DONE) break;
+      const Dec d = decode(item);
+      const int rows_b = d.rows[b];
+      if (rows_b == 0) continue;
+      mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QFULL);
+      ++wt.q[b];
+      if (r < rows_b) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)wi * (D / 2));
+      fence_proxy_async_smem();
+      mbar_arrive(&mi.q_rot[b]);
+      float m_used, l_run;
+      wg_flash_loop<D>(cx, wt, b, tS, tO, d.n, prm.scale_log2,
+                       [&](int jj) {
+                         if (jj >= d.n_cache) return wi + 1;                       // window tile: causal
+                         const int left = prm.Nk - (d.j0 + jj) * TILE;             // ragged last cache tile
+                         return left < TILE ? left : TILE;
+                       },
+                       m_used, l_run);
+      if (r == 0) mbar_arrive(&mi.q_free[b]);                 // all MMAs that read sQ[b] have completed
+      const int g = d.g0 + (b * TILE + r) / prm.w;
+      const int h = d.hkv * G + g;
+      const bool valid = r < rows_b;
+      if (prm.n_split == 1) {
+        const float inv_l = 1.0f / l_run;
+        uint4* dst = reinterpret_cast<uint4*>(prm.out + (((size_t)d.seq * prm.w + wi) * prm.Hq + h) * D);
+#pragma unroll
+        for (int q = 0; q < D / 32; ++q) {
+          uint32_t o[32];
+          tmem_ld32(tO + q * 32, o);
+          tmem_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int g4 = 0; g4 < 4; ++g4) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                pk[e] = pack_bf16x2(__uint_as_float(o[g4 * 8 + 2 * e]) * inv_l, __uint_as_float(o[g4 * 8 + 2 * e + 1]) * inv_l);
+              dst[q * 4 + g4] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+          }
+        }
+        if (valid && prm.lse_out)
+          prm.lse_out[((size_t)d.seq * prm.Hq + h) * prm.w + wi] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+      } else {
+        const size_t prow = (((size_t)d.seq * prm.Hq + h) * prm.n_split + d.split) * prm.w + wi;
+        uint4* dst = reinterpret_cast<uint4*>(prm.part_o + prow * D);
+#pragma unroll
+        for (int q = 0; q < D / 32; ++q) {
+          uint32_t o[32];
+          tmem_ld32(tO + q * 32, o);
+          tmem_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int g4 = 0; g4 < 8; ++g4) dst[q * 8 + g4] = make_uint4(o[g4 * 4], o[g4 * 4 + 1], o[g4 * 4 + 2], o[g4 * 4 + 3]);
+          }
+        }
+        if (valid) reinterpret_cast<float2*>(prm.part_ml)[prow] = make_float2(m_used, l_run);
+      }
+      tc_fence_before_sync();
+      mbar_arrive(&mi.acc_free[b]);
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == WARP_MMA) {
+    tc_fence_after_sync();
+    tmem_dealloc(cx.tmem, 512);
+  }
+}
+
+// Merge of the key splits: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  One warp per output row.
+template <int D>
+__global__ void __launch_bounds__(256) parallel_merge_kernel(const float* __restrict__ part_o,
+                                                             const float* __restrict__ part_ml, int n_rows_bh, int w,
+                                                             int Hq, int n_split, __nv_bfloat16* __restrict__ out,
+                                                             float* __restrict__ lse_out) {
+  const int row = blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5);      // (seq * Hq + h) * w + i
+  const int lane = threadIdx.x & 31;
+  if (row >= n_rows_bh * w) return;
+  const int bh = row / w, i = row % w;
+  const int seq = bh / Hq, h = bh % Hq;
+  float M = -INFINITY;
+  for (int s = 0; s < n_split; ++s) M = fmaxf(M, part_ml[(((size_t)bh * n_split + s) * w + i) * 2]);
+  float denom = 0.0f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < n_split; ++s) {
+    const size_t prow = ((size_t)bh * n_split + s) * w + i;
+    const float wgt = exp2f(part_ml[prow * 2] - M);
+    denom += wgt * part_ml[prow * 2 + 1];
+    if (lane < D / 4) {
+      const float4 o = reinterpret_cast<const float4*>(part_o + prow * D)[lane];
+      acc.x += wgt * o.x; acc.y += wgt * o.y; acc.z += wgt * o.z; acc.w += wgt * o.w;
+    }
+  }
+  const float inv = 1.0f / denom;
+  if (lane < D / 4) {
+    uint2 pk;
+    pk.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+    pk.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+    reinterpret_cast<uint2*>(out + (((size_t)seq * w + i) * Hq + h) * D)[lane] = pk;
+  }
+  if (lane == 0 && lse_out) lse_out[(size_t)bh * w + i] = (M + log2f(denom)) * 0.6931471805599453f;
 }
 
 // ====================================================================================
@@ -618,6 +883,31 @@ static cudaError_t launch_prefill_t(const CUtensorMap* maps, const PrefillParams
 
 cudaError_t launch_prefill_attn(const CUtensorMap* maps, const PrefillParams& prm, int d, int grid, cudaStream_t st) {
   return d == 128 ? launch_prefill_t<128>(maps, prm, grid, st) : launch_prefill_t<64>(maps, prm, grid, st);
+}
+
+template <int D>
+static cudaError_t launch_parallel_t(const CUtensorMap* maps, const ParallelParams& prm, int grid, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(parallel_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Cfg<D>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  parallel_attn_kernel<D><<<grid, NUM_THREADS, Cfg<D>::SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (prm.n_split > 1) {
+    const int rows = prm.B * prm.Hq * prm.w;
+    parallel_merge_kernel<D><<<(rows + 7) / 8, 256, 0, st>>>(prm.part_o, prm.part_ml, prm.B * prm.Hq, prm.w, prm.Hq,
+                                                            prm.n_split, prm.out, prm.lse_out);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+cudaError_t launch_parallel_attn(const CUtensorMap* maps, const ParallelParams& prm, int d, int grid, cudaStream_t st) {
+  return d == 128 ? launch_parallel_t<128>(maps, prm, grid, st) : launch_parallel_t<64>(maps, prm, grid, st);
 }
 
 }  // namespace pc

@@ -1,6 +1,7 @@
 // Parameter blocks and launchers of the attention kernels (internal).
 #pragma once
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <cstdint>
 
@@ -19,5 +20,22 @@ struct PrefillParams {
 
 // maps: q (box 64x1x128x1), k_rot, v, o (store), q with a w-row box
 cudaError_t launch_prefill_attn(const CUtensorMap* maps, const PrefillParams& prm, int d, int grid, cudaStream_t st);
+
+struct ParallelParams {
+  int B, w, Hq, Hkv, Nk;
+  int Gs, n_rg;                  // q-heads per row group (Gs * w <= 256), row groups per kv-head
+  int n_cache_tiles, n_split, tiles_per_split;
+  float scale_log2;
+  const double2* rope_tab;       // [w][d/2] for positions q_pos0 .. q_pos0 + w - 1
+  float* part_o;                 // [B,Hq,n_split,w,d] fp32 unnormalised partial outputs (n_split > 1)
+  float* part_ml;                // [B,Hq,n_split,w,2] (running max in log2 units, sum)
+  __nv_bfloat16* out;            // [B,w,Hq,d]
+  float* lse_out;                // [B,Hq,w] or null
+  int* status;
+  int* counter;
+};
+
+// maps: q_win (w-row box), k_cache, v_cache (128-key box), k_win, v_win (128-row box over w tokens)
+cudaError_t launch_parallel_attn(const CUtensorMap* maps, const ParallelParams& prm, int d, int grid, cudaStream_t st);
 
 }  // namespace pc
