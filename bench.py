@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the ParallelComp attention hot path on B200.
+
+One step = one pass of the whole path (chunk prefill attention with fused window scores,
+chunk ranking, token ranking, KV gather, parallel attention over the compressed cache)
+over one 128K batch of seeded synthetic input.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1] [--impl reference]
+
+N > 1 runs N independent replicas (the path has no exchange step): launch with
+torch.distributed.run; rank 0 prints the line, value = tokens of all ranks / max time.
+`--impl reference` times the CPU oracle (fp64 numpy) on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import pc_inputs  # noqa: E402
+
+METRIC = "chunked_prefill_tokens_per_s_per_layer"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def prefill_flops(cfg) -> float:
+    """Algorithmic FLOPs of the chunk-local attention: 4 d per visible (query, key) pair per q-head."""
+    return 2.0 * cfg.d * cfg.L * (cfg.L + 1) * cfg.Hq * cfg.C
+
+
+def workload_description(cfg) -> dict:
+    return {"workload": f"{cfg.name}: C={cfg.C} chunks x L={cfg.L} (ctx {cfg.ctx} + window w={cfg.w}), Hq={cfg.Hq}, "
+                        f"Hkv={cfg.Hkv}, d={cfg.d}, rope_theta={cfg.rope_theta:g}, keep m={cfg.m} chunks x k={cfg.k} "
+                        f"tokens per kv-head",
+            "tokens_per_step": cfg.C * cfg.L, "l2": "inputs (1.6 GB) larger than L2, no flush needed",
+            "parallelism": "single GPU (replicas only for N > 1)"}
+
+
+# --------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(cfg, threads_hint=None):
+    """Time the oracle, as it stands, on a bounded sample of the workload: one chunk and a
+    quarter of the head groups, full chunk length, the whole path.  Returns (tokens/s equivalent,
+    seconds, description)."""
+    from oracle import parallelcomp_oracle as orc
+    hkv_s = max(1, cfg.Hkv // 4)
+    sub = dataclasses.replace(cfg, C=1, Hq=hkv_s * cfg.G, Hkv=hkv_s, m=1, n_planted_chunks=1, planted_chunks=())
+    inp = pc_inputs.make_prefill_inputs(sub)
+    t0 = time.perf_counter()
+    orc.hot_path(inp["q"], inp["k"], inp["v"], w=sub.w, theta=sub.rope_theta, m=1, k=min(sub.k, sub.ctx))
+    dt = time.perf_counter() - t0
+    frac = (1.0 / cfg.C) * (hkv_s / cfg.Hkv)
+    tokens_equiv = cfg.C * cfg.L * frac
+    desc = (f"whole path on 1 of {cfg.C} chunks x {hkv_s} of {cfg.Hkv} kv-head groups at full L={cfg.L} "
+            f"({frac:.4g} of the step); tokens/s = {tokens_equiv:.0f} token-equivalents / {dt:.1f} s")
+    return tokens_equiv / dt, dt, desc
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        return int(n)
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals, secs, desc = [], [], ""
+    for _ in range(args.warmup_ref):
+        oracle_sample(cfg)
+    for _ in range(args.steps_ref):
+        v, s, desc = oracle_sample(cfg)
+        vals.append(v)
+        secs.append(s)
+    value = statistics.mean(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps_ref, "warmup": args.warmup_ref, "ms_per_step": 1e3 * statistics.mean(secs),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_description(cfg),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.uuid = uuid
+        self.proc = None
+        self.tmp = None
+
+    def start(self):
+        try:
+            self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", self.uuid], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        rows = [r.strip().split(",") for r in self.tmp.read().strip().splitlines() if r.strip()]
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        sm, reasons, mx, pw = [], set(), None, []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                r = [x.strip() for x in r]
+                sm.append(float(r[0]))
+                mx = float(r[1])
+                pw.append(float(r[2]))
+                for name, flag in zip(names, r[4:8]):
+                    if flag.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        if sm:
+            out.update({"sm_mhz": statistics.median(sm), "sm_max_mhz": mx, "reasons": sorted(reasons),
+                        "samples": len(sm), "power_w_max": max(pw) if pw else None})
+        return out
+
+
+# --------------------------------------------------------------------------------------- GPU leg
+def run_gpu(args, cfg):
+    import torch
+    import paper_2502_14317_b200 as pc
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    pc.load_library()
+    peaks = load_peaks()
+
+    # ---- inputs: generated once on the host (same generator the parity tests use), pinned
+    inp = pc_inputs.make_prefill_inputs(cfg, seed=cfg.seed + rank)
+
+    def pinned(bits):
+        return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+
+    hq, hk, hv = pinned(inp["q"]), pinned(inp["k"]), pinned(inp["v"])
+    q, k, v = (t.to(dev, non_blocking=True) for t in (hq, hk, hv))
+    torch.cuda.synchronize()
+    buffers: dict = {}
+    L, w = cfg.L, cfg.w
+
+    def step(events=None):
+        """The five C-ABI calls chained on the current stream (plus the stand-in chunk score)."""
+        pre = pc.chunk_prefill_attn(q, k, v, w=w, rope_theta=cfg.rope_theta, out=buffers.get("o"),
+                                    k_rot=buffers.get("k_rot"), win_score=buffers.get("win_score"),
+                                    win_lse=buffers.get("win_lse"), status=buffers.get("status"),
+                                    workspace=buffers.get("ws_prefill"))
+        if events: events[1].record()
+        score = pc.chunk_score_from_lse(pre["win_lse"], out=buffers.get("chunk_score"))
+        kept = pc.select_chunks(score, cfg.m, True, out=buffers.get("kept"))
+        idx = pc.select_tokens(pre["win_score"], kept, L - w, cfg.k, out=buffers.get("idx"))
+        if events: events[2].record()
+        kc, vc, pos = pc.gather_kv(pre["k_rot"], v, kept, idx, k_out=buffers.get("kc"), v_out=buffers.get("vc"),
+                                   pos_out=buffers.get("pos"))
+        if events: events[3].record()
+        pa = pc.parallel_attn(q[0:1, L - w:], kc.unsqueeze(0), vc.unsqueeze(0), pre["k_rot"][0:1, L - w:],
+                              v[0:1, L - w:], q_pos0=L - w, rope_theta=cfg.rope_theta, out=buffers.get("fg"),
+                              status=pre["status"], workspace=buffers.get("ws_par"))
+        buffers.update(o=pre["o"], k_rot=pre["k_rot"], win_score=pre["win_score"], win_lse=pre["win_lse"],
+                       status=pre["status"], ws_prefill=pre["workspace"], chunk_score=score, kept=kept, idx=idx,
+                       kc=kc, vc=vc, pos=pos, fg=pa["out"], ws_par=pa["workspace"])
+        return pa["out"]
+
+    # kernels launched by one step: rope table, rope keys, prefill attention, chunk score, chunk top-m,
+    # token top-k, gather, rope table (window), parallel attention, split merge
+    n_split_merge = 1 if pc.parallel_attn_workspace_bytes(1, w, cfg.Hq, cfg.Hkv, cfg.d, cfg.m * cfg.k) > 65536 else 0
+    launches_per_step = 9 + n_split_merge
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    assert int(buffers["status"].item()) == 0, "a device-side wait ran out during warm-up"
+
+    props = torch.cuda.get_device_properties(dev)
+    sampler = ClockSampler("GPU-" + str(props.uuid)) if rank == 0 else None
+    if sampler: sampler.start()
+
+    # ---- timed region: K steps, inputs resident in HBM
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for s in range(args.steps):
+        ev[s][0].record()
+        step(ev[s])
+        ev[s][4].record()
+    t_end.record()
+    barrier()
+    total_ms = t_start.elapsed_time(t_end)
+    clocks = sampler.stop() if sampler else None
+    assert int(buffers["status"].item()) == 0, "a device-side wait ran out"
+
+    stage_ms = {name: statistics.mean(ev[s][a].elapsed_time(ev[s][b]) for s in range(args.steps))
+                for name, a, b in (("prefill_attn", 0, 1), ("score_select", 1, 2), ("gather", 2, 3), ("parallel_attn", 3, 4))}
+
+    # ---- end to end through the public API with host buffers: H2D of Q,K,V and D2H of the result every step
+    e2e_steps = max(1, min(args.steps, 5))
+    h_out = torch.empty((1, w, cfg.Hq, cfg.d), dtype=torch.bfloat16).pin_memory()
+
+    def e2e_step():
+        q.copy_(hq, non_blocking=True)
+        k.copy_(hk, non_blocking=True)
+        v.copy_(hv, non_blocking=True)
+        out = step()
+        h_out.copy_(out, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    # ---- max over ranks
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(times[0]), float(times[1])
+    ms_per_step = total_ms / args.steps
+    tokens = cfg.C * cfg.L
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    if rank == 0:
+        flops = prefill_flops(cfg)
+        ach_tflops = flops / (stage_ms["prefill_attn"] * 1e-3) / 1e12
+        gather_bytes = 2.0 * (2 * cfg.Hkv * cfg.m * cfg.k * cfg.d * 2)
+        sel_bytes = 4.0 * cfg.m * cfg.Hkv * (cfg.ctx + cfg.k)
+        par_flops = 4.0 * cfg.d * (cfg.m * cfg.k + (w + 1) / 2) * w * cfg.Hq
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_description(cfg),
+            "clocks": clocks,
+            "e2e": {"value": world * tokens / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
+                    "d2h_bytes_per_step": int(h_out.numel()) * 2, "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": {"bound": "tensor", "kernel": "prefill_attn_kernel (+ RoPE pre-pass inside the same call)",
+                         "achieved": ach_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "frac": ach_tflops / peaks["bf16_tflops_sustained"],
+                         "frac_of_burst_peak": ach_tflops / peaks["bf16_tflops"],
+                         "frac_of_nominal_2250": ach_tflops / 2250.0,
+                         "peak_source": peaks["source"] + " cuBLAS bf16, sustained (kernel timed inside a long step)",
+                         "algorithmic_flops_per_launch": flops, "ms_per_launch": stage_ms["prefill_attn"],
+                         "traffic": args.traffic_bytes},
+            "stages": {
+                "prefill_attn": {"ms": stage_ms["prefill_attn"], "tflops": ach_tflops},
+                "score_select": {"ms": stage_ms["score_select"], "algorithmic_bytes": sel_bytes,
+                                 "gbs": sel_bytes / (stage_ms["score_select"] * 1e-3) / 1e9,
+                                 "note": "three launches (chunk score, chunk top-m, token top-k); latency-bound at this size"},
+                "gather": {"ms": stage_ms["gather"], "algorithmic_bytes": gather_bytes,
+                           "gbs": gather_bytes / (stage_ms["gather"] * 1e-3) / 1e9,
+                           "frac_of_measured_hbm": gather_bytes / (stage_ms["gather"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                "parallel_attn": {"ms": stage_ms["parallel_attn"],
+                                  "tflops": par_flops / (stage_ms["parallel_attn"] * 1e-3) / 1e12},
+            },
+        }
+        if not args.no_cpu_baseline and world == 1:
+            v_cpu, s_cpu, desc = oracle_sample(cfg)
+            line["cpu_baseline"] = {"value": v_cpu, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                    "sample": desc}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--chunks", type=int, default=None,
+                    help="override the number of chunks (smaller case of the same workload, e.g. for an ncu capture)")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="dram bytes per launch of the dominant kernel from an ncu capture (see profiles/)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = pc_inputs.get_config(args.workload)
+    if args.chunks is not None:
+        cfg = dataclasses.replace(cfg, name=f"{cfg.name}[C={args.chunks}]", C=args.chunks, m=min(cfg.m, args.chunks),
+                                  n_planted_chunks=min(cfg.n_planted_chunks, args.chunks))
+    if args.impl == "reference":
+        # the oracle takes ~20 s per sample: bound the run to a few minutes whatever K and W say
+        args.steps_ref = max(1, min(args.steps, 3))
+        args.warmup_ref = max(0, min(args.warmup, 1))
+        run_reference(args, cfg)
+    else:
+        run_gpu(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
