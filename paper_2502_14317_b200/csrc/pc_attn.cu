@@ -179,14 +179,14 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_taddr, uint32_t o_taddr,
     m_used = m_new;
   }
   if (!first_tile && __any_sync(0xFFFFFFFFu, raise)) {           // warp-uniform: each warp owns its 32 lanes of O
-#pragma unroll
-    for (int q = 0; q < D / 32; ++q) {
-      uint32_t o[32];
-      tmem_ld32(o_taddr + q * 32, o);
+#pragma unroll 1
+    for (int q = 0; q < D / 8; ++q) {                             // rare path: small chunks keep registers free
+      uint32_t o[8];
+      tmem_ld8(o_taddr + q * 8, o);
       tmem_wait_ld();
 #pragma unroll
-      for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-      tmem_st32(o_taddr + q * 32, o);
+      for (int j = 0; j < 8; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+      tmem_st8(o_taddr + q * 8, o);
     }
   }
   const float neg_m = (m_used == -INFINITY) ? 0.0f : -m_used;     // fully masked row so far: exp2(-inf) = 0
@@ -255,6 +255,7 @@ struct Ctx {
 };
 
 __device__ __forceinline__ void init_barriers(Misc& mi) {
+#pragma unroll
   for (int b = 0; b < 2; ++b) {
     mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 128); mbar_init(&mi.q_free[b], 1);
     mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_full[b], 128); mbar_init(&mi.o_full[b], 1);
@@ -308,6 +309,7 @@ __device__ __forceinline__ void producer_ring_tile(const Ctx& cx, Waits& wt, con
 __device__ __forceinline__ void producer_drain(const Ctx& cx, const Waits& wt) {
   Misc& mi = *cx.mi;
   for (uint32_t i = (wt.kv > NS ? wt.kv - NS : 0); i < wt.kv; ++i) mbar_wait_drain(&mi.kv_full[i % NS], full_par(i / NS));
+#pragma unroll
   for (int b = 0; b < 2; ++b)
     if (wt.q[b] > 0) mbar_wait_drain(&mi.q_full[b], full_par(wt.q[b] - 1));
 }
@@ -323,8 +325,11 @@ __device__ __forceinline__ void mma_flash_pair(const Ctx& cx, Waits& wt, const b
   const uint32_t tS[2] = {cx.tmem + 0, cx.tmem + 128}, tO[2] = {cx.tmem + 256, cx.tmem + 384};
   const int n = nb[1] > nb[0] ? nb[1] : nb[0];
   // accumulators and score buffers of earlier work must have been read out
+#pragma unroll
   for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
+#pragma unroll
   for (int e = 0; e < 2; ++e) mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
+#pragma unroll
   for (int b = 0; b < 2; ++b)
     if (has[b]) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
   tc_fence_after_sync();
@@ -332,6 +337,7 @@ __device__ __forceinline__ void mma_flash_pair(const Ctx& cx, Waits& wt, const b
     const int st = wt.kv % NS;
     mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
     tc_fence_after_sync();
+#pragma unroll
     for (int b = 0; b < 2; ++b)
       if (has[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
     mma_commit(&mi.kv_free[st]);
@@ -348,6 +354,7 @@ __device__ __forceinline__ void mma_flash_pair(const Ctx& cx, Waits& wt, const b
       mbar_wait(&mi.kv_full[st_k], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
       ++wt.kv;
     }
+#pragma unroll
     for (int b = 0; b < 2; ++b) {
       if (!has[b] || j >= nb[b]) continue;
       mbar_wait(&mi.p_full[b], full_par(wt.p[b]), cx.abort_flag, cx.status, W_PFULL);
@@ -360,27 +367,29 @@ __device__ __forceinline__ void mma_flash_pair(const Ctx& cx, Waits& wt, const b
     mma_commit(&mi.kv_free[st_v]);
     if (more) mma_commit(&mi.kv_free[st_k]);
   }
+#pragma unroll
   for (int b = 0; b < 2; ++b) if (has[b]) ++wt.acc[b];
 }
 
 // softmax group: online softmax over n key tiles for this thread's row; vis(j) = visible
 // columns of tile j.  Leaves (m_used, l_run); the accumulator O_b stays in TMEM.
 template <int D, class VisFn>
-__device__ __forceinline__ void wg_flash_loop(const Ctx& cx, Waits& wt, int b, uint32_t tS, uint32_t tO, int n,
-                                              float scale_log2, VisFn vis, float& m_used, float& l_run) {
+__device__ __forceinline__ void wg_flash_loop(const Ctx& cx, uint32_t& n_s, uint32_t& n_o, int b, uint32_t tS,
+                                              uint32_t tO, int n, float scale_log2, VisFn vis, float& m_used,
+                                              float& l_run) {
   Misc& mi = *cx.mi;
   m_used = -INFINITY;
   l_run = 0.0f;
   for (int j = 0; j < n; ++j) {
-    mbar_wait(&mi.s_full[b], full_par(wt.s[b]), cx.abort_flag, cx.status, W_SFULL);
-    ++wt.s[b];
+    mbar_wait(&mi.s_full[b], full_par(n_s), cx.abort_flag, cx.status, W_SFULL);
+    ++n_s;
     tc_fence_after_sync();
     softmax_tile<D>(tS, tO, vis(j), j == 0, scale_log2, m_used, l_run);
     tc_fence_before_sync();
     mbar_arrive(&mi.p_full[b]);
   }
-  mbar_wait(&mi.o_full[b], full_par(wt.o[b]), cx.abort_flag, cx.status, W_OFULL);
-  ++wt.o[b];
+  mbar_wait(&mi.o_full[b], full_par(n_o), cx.abort_flag, cx.status, W_OFULL);
+  ++n_o;
   tc_fence_after_sync();
 }
 
@@ -433,6 +442,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int nsub = n_subitems(sch, within);
         for (int sub = 0; sub < nsub; ++sub) {
           const SubItem it = decode_sub(sch, hkv, within, sub);
+#pragma unroll
           for (int b = 0; b < 2; ++b) {
             const int h = b ? it.hB : it.hA, t = b ? it.tB : it.tA;
             if (h < 0) continue;
@@ -453,6 +463,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int u = 0; u < n_pass; ++u) {
             const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
             const int rows_total = heads * prm.w;
+#pragma unroll
             for (int b = 0; b < 2; ++b) {
               const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
               if (rows_b == 0) continue;
@@ -491,40 +502,44 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           mma_flash_pair<D>(cx, wt, has, nb);
         }
         if (within == 0) {
+#pragma unroll
           for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
           for (int u = 0; u < n_pass; ++u) {
             const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
             const int rows_total = heads * prm.w;
             const int rows[2] = {rows_total < TILE ? rows_total : TILE, rows_total > TILE ? rows_total - TILE : 0};
+#pragma unroll
             for (int b = 0; b < 2; ++b)
               if (rows[b] > 0) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
             for (int j = 0; j < sch.T; ++j) {
               const int e = j & 1;
-              mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
+              mbar_wait(&mi.t_free[e], free_par(e ? wt.t[1] : wt.t[0]), cx.abort_flag, cx.status, W_TFREE);
               const int st = wt.kv % NS;
               mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
               ++wt.kv;
               tc_fence_after_sync();
+#pragma unroll
               for (int b = 0; b < 2; ++b)
                 if (rows[b] > 0)
                   issue_kq<D>(cx.tmem + e * 256 + b * 128, ring_u32 + st * C::TILE_BYTES, q_u32[b], (rows[b] + 15) & ~15);
               mma_commit(&mi.t_full[e]);
               mma_commit(&mi.kv_free[st]);
-              ++wt.t[e];
+              if (e) ++wt.t[1]; else ++wt.t[0];
             }
           }
         }
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp < 8) {
     // ================================================================ softmax groups
     const int b = warp >> 2;                                 // block / group index
     const int r = tid & 127;                                 // row in the block = TMEM lane
     const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tS = cx.tmem + b * 128 + lane_sel, tO = cx.tmem + 256 + b * 128 + lane_sel;
     const float scale_log2 = prm.scale_log2;
-    uint8_t* const myQ = cx.sQ[b];
+    uint8_t* const myQ = b ? cx.sQ[1] : cx.sQ[0];
+    uint32_t n_q = 0, n_s = 0, n_o = 0, n_t0 = 0, n_t1 = 0;   // barrier use counts of this group
     while (true) {
       const int item = consumer_next_item(cx, wt);
       if (item == ITEM_DONE) break;
@@ -537,15 +552,15 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (h < 0) continue;
         const int token = t * TILE + r;
         // ---- Q prologue: rotate this thread's row in shared memory
-        mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QFULL);
-        ++wt.q[b];
+        mbar_wait(&mi.q_full[b], full_par(n_q), cx.abort_flag, cx.status, W_QFULL);
+        ++n_q;
         if (token < prm.L) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)token * (D / 2));
         fence_proxy_async_smem();
         mbar_arrive(&mi.q_rot[b]);
         // ---- main loop over key tiles (causal: keys <= token; only the diagonal tile is masked)
         float m_used, l_run;
         const int n = t + 1;
-        wg_flash_loop<D>(cx, wt, b, tS, tO, n, scale_log2,
+        wg_flash_loop<D>(cx, n_s, n_o, b, tS, tO, n, scale_log2,
                          [&](int j) { return (j == n - 1) ? (token - j * TILE + 1) : TILE; }, m_used, l_run);
         // ---- epilogue: normalise, stage bf16 rows in the (now idle) Q buffer, TMA store
         const float inv_l = 1.0f / l_run;
@@ -593,8 +608,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int rows_total = heads * prm.w;
           const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
           if (rows_b > 0) {
-            mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QFULL);
-            ++wt.q[b];
+            mbar_wait(&mi.q_full[b], full_par(n_q), cx.abort_flag, cx.status, W_QFULL);
+            ++n_q;
             if (r < rows_b) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)(prm.L - prm.w + (r % prm.w)) * (D / 2));
             fence_proxy_async_smem();
             mbar_arrive(&mi.q_rot[b]);
@@ -602,8 +617,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const float* lse_rows = mi.lse2 + u * Gs * prm.w + b * TILE;   // log-sum-exp of the window row on column n
           for (int j = 0; j < sch.T; ++j) {
             const int e = j & 1;
-            mbar_wait(&mi.t_full[e], full_par(wt.t[e]), cx.abort_flag, cx.status, W_TFULL);
-            ++wt.t[e];
+            mbar_wait(&mi.t_full[e], full_par(e ? n_t1 : n_t0), cx.abort_flag, cx.status, W_TFULL);
+            if (e) ++n_t1; else ++n_t0;
             tc_fence_after_sync();
             const int key = j * TILE + r;
             const bool need_mask = (j * TILE + TILE - 1) > (prm.L - prm.w);
@@ -716,6 +731,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
         const int item = producer_next_item(cx, wt, prm.counter, n_items);
         if (item == ITEM_DONE) break;
         const Dec d = decode(item);
+#pragma unroll
         for (int b = 0; b < 2; ++b) {
           if (d.rows[b] == 0) continue;
           mbar_wait(&mi.q_free[b], free_par(wt.q[b]), cx.abort_flag, cx.status, W_QFREE);
@@ -752,26 +768,27 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp < 8) {
     const int b = warp >> 2;
     const int r = tid & 127;
     const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tS = cx.tmem + b * 128 + lane_sel, tO = cx.tmem + 256 + b * 128 + lane_sel;
-    uint8_t* const myQ = cx.sQ[b];
+    uint8_t* const myQ = b ? cx.sQ[1] : cx.sQ[0];
+    uint32_t n_q = 0, n_s = 0, n_o = 0;
     const int wi = r % prm.w;                                 // window index of this row (128 % w == 0)
     while (true) {
       const int item = consumer_next_item(cx, wt);
       if (item == ITEM_DONE) break;
       const Dec d = decode(item);
-      const int rows_b = d.rows[b];
+      const int rows_b = b ? d.rows[1] : d.rows[0];
       if (rows_b == 0) continue;
-      mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QFULL);
-      ++wt.q[b];
+      mbar_wait(&mi.q_full[b], full_par(n_q), cx.abort_flag, cx.status, W_QFULL);
+      ++n_q;
       if (r < rows_b) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)wi * (D / 2));
       fence_proxy_async_smem();
       mbar_arrive(&mi.q_rot[b]);
       float m_used, l_run;
-      wg_flash_loop<D>(cx, wt, b, tS, tO, d.n, prm.scale_log2,
+      wg_flash_loop<D>(cx, n_s, n_o, b, tS, tO, d.n, prm.scale_log2,
                        [&](int jj) {
                          if (jj >= d.n_cache) return wi + 1;                       // window tile: causal
                          const int left = prm.Nk - (d.j0 + jj) * TILE;             // ragged last cache tile
