@@ -160,6 +160,21 @@ class ClockSampler:
         return out
 
 
+# --------------------------------------------------------------------------------------- replicas
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of per-rank timings over all ranks (identity for a single process)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def replica_throughput(units_per_rank: float, world: int, max_ms_per_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas: all units / slowest rank's time."""
+    return world * units_per_rank / (max_ms_per_step * 1e-3)
+
+
 # --------------------------------------------------------------------------------------- GPU leg
 def run_gpu(args, cfg):
     import torch
@@ -272,13 +287,10 @@ def run_gpu(args, cfg):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # ---- max over ranks
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(times[0]), float(times[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, dev)
     ms_per_step = total_ms / args.steps
     tokens = cfg.C * cfg.L
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = replica_throughput(tokens, world, ms_per_step)
 
     if rank == 0:
         flops = prefill_flops(cfg)
@@ -292,7 +304,7 @@ def run_gpu(args, cfg):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": workload_description(cfg),
             "clocks": clocks,
-            "e2e": {"value": world * tokens / (e2e_ms * 1e-3), "unit": UNIT,
+            "e2e": {"value": replica_throughput(tokens, world, e2e_ms), "unit": UNIT,
                     "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
                     "d2h_bytes_per_step": int(h_out.numel()) * 2, "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches_per_step * args.steps,

@@ -25,8 +25,8 @@
  *     whose bounded wait on a copy or tensor-core barrier ran out stores a non-zero
  *     code there and the results of that call are undefined.  The caller clears it and
  *     reads it after synchronising.  No kernel spins without a limit.
- *   - Supported: d in {64, 128}; Hq % Hkv == 0; w % 8 == 0; 8 <= w <= 128; w < L;
- *     G * w <= 256 rows are handled per pass (larger groups take several passes).
+ *   - Supported: d in {64, 128}; Hq % Hkv == 0; w a power of two in [8, 128]; w < L;
+ *     G * w <= 1024 (256 window rows are handled per pass, larger groups take several).
  */
 #ifndef PC_H_
 #define PC_H_

@@ -1,0 +1,116 @@
+"""CPU-only checks of the boundary and host logic: the library loads and exports every symbol that
+include/pc.h declares; host-side argument validation; bench.py's replica aggregation over gloo."""
+import ctypes
+import json
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2502_14317_b200 import build, binding
+    build.build_library()
+    return binding.load_library()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "pc.h")).read()
+    return sorted(set(re.findall(r"PC_API\s+[\w\s\*]+?\b(pc_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert set(names) >= {"pc_chunk_prefill_attn", "pc_select_chunks", "pc_select_tokens", "pc_gather_kv",
+                          "pc_parallel_attn", "pc_chunk_prefill_attn_workspace_bytes",
+                          "pc_parallel_attn_workspace_bytes", "pc_chunk_score_from_lse", "pc_status_string",
+                          "pc_version"}
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in pc.h but not exported by libpc.so"
+
+
+def test_status_strings_and_version(lib):
+    from paper_2502_14317_b200 import binding
+    assert binding.version() >= 1000
+    assert binding.status_string(0) == "ok"
+    texts = {binding.status_string(c) for c in (-1, -2, -3, -4, -5)}
+    assert len(texts) == 5 and "unknown status" not in texts
+    assert binding.status_string(-99) == "unknown status"
+
+
+def test_workspace_queries_are_host_only(lib):
+    from paper_2502_14317_b200 import binding
+    # cfg1: 256 B counter + fp64 cos/sin table L * d/2 * 16 B
+    assert binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128) == 256 + 8192 * 64 * 16
+    with_krot = binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128, k_rot_in_workspace=True)
+    assert with_krot == 256 + 8192 * 64 * 16 + 16 * 8192 * 8 * 128 * 2
+    # unsupported shapes give 0
+    assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 24, 4, 2, 64) == 0       # window not a power of two
+    assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 2, 96) == 0       # head size
+    assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 3, 64) == 0       # Hq % Hkv
+    assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 128, 16384) > 0
+    assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 100, 16384) == 0
+
+
+def test_host_side_argument_errors_need_no_gpu(lib):
+    # null pointers / bad sizes are rejected before any CUDA call
+    assert lib.pc_select_chunks(None, 4, 2, 1, None, None) == -1
+    buf = (ctypes.c_float * 4)()
+    out = (ctypes.c_int32 * 4)()
+    p, o = ctypes.cast(buf, ctypes.c_void_p), ctypes.cast(out, ctypes.c_void_p)
+    assert lib.pc_select_chunks(p, 4, 5, 1, o, None) == -1          # m > C
+    assert lib.pc_select_chunks(p, 2000, 5, 1, o, None) == -2       # C > 1024
+    assert lib.pc_select_tokens(p, o, 4, 2, 2, 256, 300, 64, o, None) == -1    # n_cand > L
+    assert lib.pc_gather_kv(p, p, None, 256, o, o, 2, 2, 64, 96, p, p, None, None) == -2   # head size
+    assert lib.pc_parallel_attn(1, 24, 4, 2, 64, 128, p, 0, 1e4, 0.0, p, p, p, p, p, None, None, None, 0, None) == -2
+
+
+def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
+    from paper_2502_14317_b200 import binding
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "lib_path", lambda: str(tmp_path / "missing.so"))
+    with pytest.raises(binding.PcError, match="no fallback"):
+        binding.load_library()
+
+
+_WORKER = r"""
+import os, sys, json
+sys.path.insert(0, {root!r})
+import torch.distributed as dist
+import bench
+dist.init_process_group("gloo", rank=int(os.environ["RANK"]), world_size=2)
+rank = dist.get_rank()
+total_ms, e2e_ms = bench.max_over_ranks([10.0 + 5.0 * rank, 40.0 - 3.0 * rank], dist)
+value = bench.replica_throughput(131072, dist.get_world_size(), total_ms / 1)
+if rank == 0:
+    print(json.dumps({{"total_ms": total_ms, "e2e_ms": e2e_ms, "value": value}}))
+dist.barrier()
+dist.destroy_process_group()
+"""
+
+
+def test_replica_aggregation_world_size_2_gloo(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(_WORKER.format(root=ROOT))
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT="29577")
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    outs = [p.communicate(timeout=120) for p in procs]
+    assert all(p.returncode == 0 for p in procs), outs
+    res = json.loads(outs[0][0].strip().splitlines()[-1])
+    assert res["total_ms"] == 15.0 and res["e2e_ms"] == 40.0           # slowest rank on each clock
+    assert abs(res["value"] - 2 * 131072 / 15e-3) < 1e-6               # all ranks' tokens / slowest time
+
+
+def test_reference_arm_other_ranks_do_nothing():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
+                       env=env, capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0 and r.stdout.strip() == ""
