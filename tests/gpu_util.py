@@ -23,7 +23,10 @@ def check_attention_output(got_f64: np.ndarray, ref: np.ndarray, what: str = "O"
 
     Pure relative error is meaningless near zero and the bf16 output grid alone exceeds
     1e-2 absolute for |x| > 4, so the element-wise gate is |d| <= 1e-2 + 2e-2 |ref|; the
-    two raw maxima are checked on the ranges where each is meaningful.
+    two raw maxima are checked on the ranges where each is meaningful.  The tensor-core path
+    rounds the probabilities to bf16 (unit round-off 2^-9), which bounds the error of an output
+    by 2^-9 * sum_j A_ij |v_j| <= 2^-9 * max|v| (about 1e-2 for |v| up to 5); a relative bound of
+    2e-2 therefore follows from the arithmetic only where |ref| >= 2^-9 * max|v| / 2e-2 ~ 0.5.
     """
     d = np.abs(got_f64 - ref)
     assert np.all(np.isfinite(got_f64)), f"{what}: non-finite values"
@@ -32,10 +35,10 @@ def check_attention_output(got_f64: np.ndarray, ref: np.ndarray, what: str = "O"
     small = np.abs(ref) <= 1.0
     if small.any():
         assert d[small].max() <= 1e-2, f"{what}: max-abs {d[small].max():.4e} on |ref| <= 1"
-    big = np.abs(ref) >= 0.1
+    big = np.abs(ref) >= 0.5
     if big.any():
         rel = (d[big] / np.abs(ref[big])).max()
-        assert rel <= 2e-2, f"{what}: max-rel {rel:.4e} on |ref| >= 0.1"
+        assert rel <= 2e-2, f"{what}: max-rel {rel:.4e} on |ref| >= 0.5"
     return float(d.max())
 
 
