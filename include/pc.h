@@ -50,7 +50,8 @@ typedef enum {
   PC_ERR_UNSUPPORTED = -2,   /* shape outside the supported set, or device is not sm_100  */
   PC_ERR_WORKSPACE = -3,     /* workspace missing or smaller than *_workspace_bytes       */
   PC_ERR_CUDA = -4,          /* a CUDA runtime / driver call failed                       */
-  PC_ERR_TIMEOUT = -5        /* value stored in status_word by a kernel whose wait ran out */
+  PC_ERR_TIMEOUT = -5,       /* value stored in status_word by a kernel whose wait ran out */
+  PC_ERR_SCRATCH_LIMIT = -6  /* pc_parallel_attn_static: the shape needs more than PC_STATIC_SCRATCH_BYTES */
 } pc_status;
 
 /* Text for a status code (static storage). */
@@ -154,6 +155,46 @@ PC_API int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, i
                          const void* k_cache, const void* v_cache, const void* k_win, const void* v_win,
                          void* out, float* lse_out, int32_t* status_word, void* workspace,
                          size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * pc_parallel_attn without a workspace argument, for callers that must not allocate.
+ * The paper has no counterpart of this call: it computes exactly what pc_parallel_attn
+ * computes (same kernels, same split plan, same results) and exists for the callers
+ * below.
+ *
+ * Who needs it: code that runs where device allocation is off limits at call time -
+ * an inference server that sized all of its memory at start-up and treats a later
+ * cudaMalloc as a bug, a component embedded in a host application that owns the
+ * allocator, a real-time loop that cannot take the implicit device synchronisation an
+ * allocation may cause.  Such callers can still pass inputs and outputs they already
+ * hold, but have nowhere to get a workspace from.
+ *
+ * The scratch (work counter, window cos/sin table, per-split partial results) is a
+ * fixed array of PC_STATIC_SCRATCH_BYTES inside the library image.  Consequences:
+ *   - every GPU on which the library is loaded gives up that much memory until the
+ *     process exits, whether or not this call is ever used;
+ *   - a shape whose pc_parallel_attn_workspace_bytes exceeds the array is refused with
+ *     PC_ERR_SCRATCH_LIMIT before anything is launched (B = 1 with tens of thousands of
+ *     cached keys splits widely and can exceed it; batches of sequences need little);
+ *   - all calls on a device share the one array and it keeps whatever the previous
+ *     call left there.  The call clears the part that has to start at zero (the work
+ *     counter) on `stream` itself.  Two calls whose kernels can overlap on the GPU
+ *     (different streams, or different host threads on different streams) race on the
+ *     array: serialise them on one stream or with events;
+ *   - the first call on each device looks up the array's device address (a host-side
+ *     query, no allocation, no launch).  Make that first call outside of any stream
+ *     capture; later calls on that device skip the query.
+ * The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ * Arguments, layouts, status word and return values otherwise as for pc_parallel_attn.
+ */
+#define PC_STATIC_SCRATCH_BYTES (16u << 20)
+
+PC_API size_t pc_parallel_attn_static_scratch_bytes(void);
+
+PC_API int32_t pc_parallel_attn_static(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk,
+                                const void* q_win, int32_t q_pos0, float rope_theta, float softmax_scale,
+                                const void* k_cache, const void* v_cache, const void* k_win, const void* v_win,
+                                void* out, float* lse_out, int32_t* status_word, void* stream);
 
 #ifdef __cplusplus
 }

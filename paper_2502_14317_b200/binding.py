@@ -62,6 +62,10 @@ def load_library():
     lib.pc_parallel_attn.restype = c_int32
     lib.pc_parallel_attn.argtypes = [c_int32] * 6 + [c_void_p, c_int32, c_float, c_float] + [c_void_p] * 8 + \
                                     [c_size_t, c_void_p]
+    lib.pc_parallel_attn_static_scratch_bytes.restype = c_size_t
+    lib.pc_parallel_attn_static_scratch_bytes.argtypes = []
+    lib.pc_parallel_attn_static.restype = c_int32
+    lib.pc_parallel_attn_static.argtypes = [c_int32] * 6 + [c_void_p, c_int32, c_float, c_float] + [c_void_p] * 8
     _LIB = lib
     return lib
 
@@ -227,6 +231,36 @@ def parallel_attn(q_win, k_cache, v_cache, k_win, v_win, *, q_pos0, rope_theta, 
                               _ptr(status), _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "pc_parallel_attn")
     return {"out": out, "lse": lse_out, "status": status, "workspace": workspace}
+
+
+def parallel_attn_static_scratch_bytes() -> int:
+    return int(load_library().pc_parallel_attn_static_scratch_bytes())
+
+
+def parallel_attn_static(q_win, k_cache, v_cache, k_win, v_win, out, *, q_pos0, rope_theta, softmax_scale=0.0,
+                         lse_out=None, status=None):
+    """pc_parallel_attn_static: pc_parallel_attn for callers that may not allocate device memory.
+
+    Nothing is allocated here either: ``out`` (and ``lse_out`` / ``status`` if wanted) must be passed in, and
+    the scratch is the fixed array inside the library.  Shapes that need more scratch than that array
+    holds are refused.  Calls on one device share the array, so keep them on one stream.
+    """
+    lib = load_library()
+    _need_cuda(q_win, k_cache, v_cache, k_win, v_win, out)
+    B, w, Hq, d = q_win.shape
+    Hkv, Nk = k_cache.shape[1], k_cache.shape[2]
+    for t in (q_win, k_cache, v_cache, k_win, v_win, out):
+        if not t.is_contiguous():
+            raise PcError("pc_parallel_attn_static takes contiguous tensors")
+    need, have = parallel_attn_workspace_bytes(B, w, Hq, Hkv, d, Nk), parallel_attn_static_scratch_bytes()
+    if need > have:
+        raise PcError(f"pc_parallel_attn_static: this shape needs {need} bytes of scratch, the built-in array holds "
+                      f"{have}; use pc_parallel_attn with a workspace instead")
+    rc = lib.pc_parallel_attn_static(B, w, Hq, Hkv, d, Nk, _ptr(q_win), int(q_pos0), float(rope_theta),
+                                     float(softmax_scale), _ptr(k_cache), _ptr(v_cache), _ptr(k_win), _ptr(v_win),
+                                     _ptr(out), _ptr(lse_out), _ptr(status), _stream())
+    _check(rc, "pc_parallel_attn_static")
+    return out
 
 
 def hot_path(q, k, v, *, w, rope_theta, m, k_keep, softmax_scale=0.0, chunk_score=None, buffers=None):

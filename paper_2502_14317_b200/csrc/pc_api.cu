@@ -79,6 +79,7 @@ const char* pc_status_string(int32_t status) {
     case PC_ERR_WORKSPACE: return "workspace missing or too small";
     case PC_ERR_CUDA: return "CUDA call failed";
     case PC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case PC_ERR_SCRATCH_LIMIT: return "shape needs more scratch than the built-in PC_STATIC_SCRATCH_BYTES array holds";
     default: return "unknown status";
   }
 }
