@@ -1,11 +1,17 @@
 // Attention kernels for sm_100a: chunk-local causal attention with fused query-window
 // scores (Eq. 1-2, Eq. 5-6) and parallel attention over the compressed cache (Eq. 9-11).
 //
-// One persistent CTA per SM, 10 warps:
+// One persistent CTA per SM, 12 warps in 3 warpgroups:
 //   warps 0-3  softmax group 0   (one 128-row query block, thread = row = TMEM lane)
 //   warps 4-7  softmax group 1   (a second 128-row block sharing the same K/V tiles)
 //   warp  8    TMA producer      (Q tiles, K/V ring)
-//   warp  9    tcgen05 issuer    (owns TMEM allocation)
+//   warp  9    tcgen05 issuer for block 0 (owns the TMEM allocation)
+//   warp 10    tcgen05 issuer for block 1
+//   warp 11    idle
+// Two issuers, not one: a tcgen05.mma issue blocks while the tensor pipe is busy, and every
+// barrier wait or commit between two batches costs the issuing thread ~100 cycles during
+// which a single issuer lets the pipe run dry.  With one issuer per block the waits of one
+// overlap the issue of the other.
 // Per 128-key tile:  S_b = Q_b K^T  (SS MMA, fp32 in TMEM)  ->  softmax group b turns S_b
 // into bf16 P_b in place in TMEM  ->  O_b += P_b V  (TS MMA, V as N-major smem operand).
 // While group 0 runs its softmax the tensor core works for group 1 and vice versa.
@@ -21,27 +27,37 @@
 #include "pc_attn.h"
 #include "pc_sm100.cuh"
 
+#ifndef PC_SETMAXNREG
+#define PC_SETMAXNREG 0
+#endif
+#ifndef PC_POLY_PAIRS_PER_8
+#define PC_POLY_PAIRS_PER_8 2
+#endif
+
 namespace pc {
 
 namespace {
 
 constexpr int TILE = 128;
-constexpr int NUM_THREADS = 320;
+constexpr int NUM_THREADS = 384;               // 3 warpgroups: softmax 0, softmax 1, {producer, issuer, 2 idle warps}
+constexpr int REGS_SOFTMAX = 224, REGS_SERVICE = 56;   // per-thread registers after re-partitioning (sum <= 64 K)
 constexpr int WARP_PRODUCER = 8;
-constexpr int WARP_MMA = 9;
+constexpr int WARP_MMA = 9;                 // issuer of block 0; WARP_MMA + 1 issues block 1
 constexpr int NS = 4;                       // K/V ring stages
 constexpr float LAZY_RESCALE = 8.0f;        // log2 units
 constexpr int ITEM_DONE = -1;
+constexpr int POLY_PAIRS_PER_8 = PC_POLY_PAIRS_PER_8;   // of every 8 logit pairs, how many take the polynomial exp2
 
 // where-codes stored in the status word when a wait gives up
-enum { W_ITEM = 101, W_QFULL, W_QROT, W_QFREE, W_KVFULL, W_KVFREE, W_SFULL, W_PFULL, W_OFULL, W_ACCFREE, W_TFULL, W_TFREE };
+enum { W_ITEM = 101, W_QFULL, W_QROT, W_QFREE, W_KVFULL, W_KVFREE, W_SFULL, W_PFULL, W_OFULL, W_ACCFREE, W_TFULL, W_TFREE, W_TURN, W_PHALF };
 
 struct __align__(16) Misc {
   uint64_t q_full[2], q_rot[2], q_free[2];
   uint64_t kv_full[NS], kv_free[NS];
-  uint64_t s_full[2], p_full[2], o_full[2], acc_free[2];
+  uint64_t s_full[2], p_half[2], p_full[2], o_full[2], acc_free[2];
   uint64_t item_full[2], item_empty[2];
   uint64_t t_full[2], t_free[2];
+  uint64_t turn[2];                        // issue token passed between the two tcgen05 issuers
   int item_slot[2];
   uint32_t tmem_base;
   int abort_flag;
@@ -148,29 +164,32 @@ __device__ __forceinline__ void rope_row_smem(uint8_t* tile, int row, const doub
 // Reads the 128 fp32 logits of this thread's row from TMEM, updates the running
 // (m, l), rescales the accumulator when the maximum moved by more than 2^LAZY_RESCALE,
 // and writes bf16 probabilities back over the logits.  `vis` = visible columns (<= 0: none).
+// The first half of the probabilities (keys 0..63) is published on `p_half_bar` as soon as it
+// is in TMEM, so that the first half of P V runs under the exponentials of the second half.
 template <int D>
 __device__ __forceinline__ void softmax_tile(uint32_t s_taddr, uint32_t o_taddr, int vis, bool first_tile,
-                                             float scale_log2, float& m_used, float& l_run) {
+                                             float scale_log2, float& m_used, float& l_run, uint64_t* p_half_bar) {
   uint32_t s[4][32];
 #pragma unroll
   for (int q = 0; q < 4; ++q) tmem_ld32(s_taddr + q * 32, s[q]);
   tmem_wait_ld();
-  float mx = -INFINITY;
-  if (vis >= TILE) {
+  if (vis < TILE) {
 #pragma unroll
     for (int q = 0; q < 4; ++q)
 #pragma unroll
-      for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(s[q][j]));
-  } else {
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        if (q * 32 + j >= vis) s[q][j] = 0xFF800000u;            // -inf
-        mx = fmaxf(mx, __uint_as_float(s[q][j]));
-      }
+      for (int j = 0; j < 32; ++j)
+        if (q * 32 + j >= vis) s[q][j] = 0xFF800000u;              // -inf
   }
-  const float m_tile = mx * scale_log2;                          // -inf if nothing visible
+  // row maximum: four independent chains of 3-input max
+  float mq[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    float a = fmax3(__uint_as_float(s[q][0]), __uint_as_float(s[q][1]), __uint_as_float(s[q][2]));
+#pragma unroll
+    for (int j = 3; j < 31; j += 2) a = fmax3(a, __uint_as_float(s[q][j]), __uint_as_float(s[q][j + 1]));
+    mq[q] = fmaxf(a, __uint_as_float(s[q][31]));
+  }
+  const float m_tile = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3])) * scale_log2;   // -inf if nothing visible
   float alpha = 1.0f;
   const bool raise = first_tile || (m_tile > m_used + LAZY_RESCALE);
   if (raise) {
@@ -190,20 +209,36 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_taddr, uint32_t o_taddr,
     }
   }
   const float neg_m = (m_used == -INFINITY) ? 0.0f : -m_used;     // fully masked row so far: exp2(-inf) = 0
-  float sum = 0.0f;
+  const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), negm2 = pack_f32x2(neg_m, neg_m);
+  uint64_t sum2[2] = {0ull, 0ull};                                // four partial row sums (two packed pairs)
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     uint32_t packed[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const float p0 = fast_exp2(fmaf(__uint_as_float(s[q][2 * j]), scale_log2, neg_m));
-      const float p1 = fast_exp2(fmaf(__uint_as_float(s[q][2 * j + 1]), scale_log2, neg_m));
-      sum += p0 + p1;
+      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[q][2 * j]), __uint_as_float(s[q][2 * j + 1])), scale2, negm2);
+      float x0, x1, p0, p1;
+      unpack_f32x2(x2, x0, x1);
+      if (((j * POLY_PAIRS_PER_8) % 8) < POLY_PAIRS_PER_8) {
+        exp2_poly_x2(x0, x1, p0, p1);                             // FMA pipe
+      } else {
+        p0 = fast_exp2(x0);                                       // MUFU pipe
+        p1 = fast_exp2(x1);
+      }
+      sum2[j & 1] = add_f32x2(sum2[j & 1], pack_f32x2(p0, p1));
       packed[j] = pack_bf16x2(p0, p1);
     }
     tmem_st16(s_taddr + q * 16, packed);                          // P aliases the first 64 columns of S
+    if (q == 1) {                                                 // keys 0..63 of P are final: the issuer may start P V on them
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(p_half_bar);
+    }
   }
-  l_run = l_run * alpha + sum;
+  float a0, a1, a2, a3;
+  unpack_f32x2(sum2[0], a0, a1);
+  unpack_f32x2(sum2[1], a2, a3);
+  l_run = l_run * alpha + ((a0 + a1) + (a2 + a3));
   tmem_wait_st();
 }
 
@@ -223,11 +258,13 @@ template <int D>
 __device__ __forceinline__ void issue_kq(uint32_t d_tmem, uint32_t k_smem, uint32_t q_smem, int n_cols) {
   issue_qk<D>(d_tmem, k_smem, q_smem, n_cols);
 }
+// k-steps [ks0, ks1) of O += P V (16 keys per step)
 template <int D>
-__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate) {
+__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate, int ks0,
+                                         int ks1) {
   constexpr uint32_t idesc = make_idesc_bf16_f32(TILE, D, false, true);
 #pragma unroll
-  for (int ks = 0; ks < TILE / 16; ++ks) {
+  for (int ks = ks0; ks < ks1; ++ks) {
     mma_ts(o_tmem, p_tmem + ks * 8, make_smem_desc_sw128(v_smem + ks * 2048, 16384, 1024), idesc,
            accumulate || ks > 0);
   }
@@ -237,8 +274,9 @@ __device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint3
 struct Waits {                                 // how many times each barrier has been used by this role
   uint32_t q[2] = {0, 0};                      // q_full / q_rot / q_free (one use per block load)
   uint32_t kv = 0;                             // ring position (monotone)
-  uint32_t s[2] = {0, 0}, p[2] = {0, 0}, o[2] = {0, 0}, acc[2] = {0, 0};
+  uint32_t s[2] = {0, 0}, p[2] = {0, 0}, o[2] = {0, 0}, acc[2] = {0, 0};   // p counts p_half and p_full alike
   uint32_t t[2] = {0, 0};
+  uint32_t turn = 0;                           // batches issued so far by this issuer
   uint32_t item = 0;
 };
 __device__ __forceinline__ uint32_t full_par(uint32_t n) { return n & 1u; }          // n-th use of a "full" barrier
@@ -258,12 +296,13 @@ __device__ __forceinline__ void init_barriers(Misc& mi) {
 #pragma unroll
   for (int b = 0; b < 2; ++b) {
     mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 128); mbar_init(&mi.q_free[b], 1);
-    mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_full[b], 128); mbar_init(&mi.o_full[b], 1);
+    mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_half[b], 128); mbar_init(&mi.p_full[b], 128); mbar_init(&mi.o_full[b], 1);
     mbar_init(&mi.acc_free[b], 128);
-    mbar_init(&mi.item_full[b], 1); mbar_init(&mi.item_empty[b], 257);
-    mbar_init(&mi.t_full[b], 1); mbar_init(&mi.t_free[b], 256);
+    mbar_init(&mi.item_full[b], 1); mbar_init(&mi.item_empty[b], 258);
+    mbar_init(&mi.t_full[b], 2); mbar_init(&mi.t_free[b], 256);
+    mbar_init(&mi.turn[b], 1);
   }
-  for (int s = 0; s < NS; ++s) { mbar_init(&mi.kv_full[s], 1); mbar_init(&mi.kv_free[s], 1); }
+  for (int s = 0; s < NS; ++s) { mbar_init(&mi.kv_full[s], 1); mbar_init(&mi.kv_free[s], 2); }   // both issuers release a stage
   mi.abort_flag = 0;
   fence_mbar_init();
 }
@@ -314,34 +353,52 @@ __device__ __forceinline__ void producer_drain(const Ctx& cx, const Waits& wt) {
     if (wt.q[b] > 0) mbar_wait_drain(&mi.q_full[b], full_par(wt.q[b] - 1));
 }
 
-// issuer: the flash loop for a pair of query blocks sharing K/V tiles.  Ring order is
-// K0, V0, K1, V1, ...; block b takes part in its first nb[b] tiles.
+// The two issuers take turns: the tensor pipe then runs the batch of one block to its end
+// before the other block's batch, which keeps the two softmax groups half a period apart
+// (while one group computes, the pipe works for the other).  Issuer 0 goes first.
+__device__ __forceinline__ void turn_take(const Ctx& cx, Waits& wt, int b) {
+  Misc& mi = *cx.mi;
+  mbar_wait(&mi.turn[b], b == 0 ? free_par(wt.turn) : full_par(wt.turn), cx.abort_flag, cx.status, W_TURN);
+}
+__device__ __forceinline__ void turn_pass(const Ctx& cx, Waits& wt, int b) {
+  mbar_arrive(&cx.mi->turn[b ^ 1]);
+  ++wt.turn;
+}
+
+// issuer of block b: the flash loop over the n K/V tiles of the ring (order K0, V0, K1, V1, ...).
+// Block b takes part in its first nb_b tiles; the issuer of an absent or shorter block still
+// walks the ring, takes its turns and releases the stages it does not use, so that both
+// issuers arrive once on every kv_free barrier and the token keeps alternating.
 template <int D>
-__device__ __forceinline__ void mma_flash_pair(const Ctx& cx, Waits& wt, const bool has[2], const int nb[2]) {
+__device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b, bool has_b, int nb_b, int n) {
   using C = Cfg<D>;
   Misc& mi = *cx.mi;
   const uint32_t ring_u32 = smem_u32(cx.ring);
-  const uint32_t q_u32[2] = {smem_u32(cx.sQ[0]), smem_u32(cx.sQ[1])};
-  const uint32_t tS[2] = {cx.tmem + 0, cx.tmem + 128}, tO[2] = {cx.tmem + 256, cx.tmem + 384};
-  const int n = nb[1] > nb[0] ? nb[1] : nb[0];
-  // accumulators and score buffers of earlier work must have been read out
+  const uint32_t q_u32 = smem_u32(cx.sQ[b]);
+  const uint32_t tS = cx.tmem + b * 128, tO = cx.tmem + 256 + b * 128;
+  if (has_b) {
+    // accumulator and score buffers of earlier work must have been read out
+    mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
 #pragma unroll
-  for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
-#pragma unroll
-  for (int e = 0; e < 2; ++e) mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
-#pragma unroll
-  for (int b = 0; b < 2; ++b)
-    if (has[b]) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
-  tc_fence_after_sync();
+    for (int e = 0; e < 2; ++e) mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
+    mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT);
+    ++wt.q[b];
+  }
   {  // S(0)
     const int st = wt.kv % NS;
     mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
-    tc_fence_after_sync();
-#pragma unroll
-    for (int b = 0; b < 2; ++b)
-      if (has[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
-    mma_commit(&mi.kv_free[st]);
     ++wt.kv;
+    turn_take(cx, wt, b);
+    if (has_b) {
+      tc_fence_after_sync();
+      issue_qk<D>(tS, q_u32, ring_u32 + st * C::TILE_BYTES, TILE);
+      mma_commit(&mi.s_full[b]);
+      turn_pass(cx, wt, b);
+      mma_commit(&mi.kv_free[st]);
+    } else {
+      turn_pass(cx, wt, b);
+      mbar_arrive(&mi.kv_free[st]);
+    }
   }
   for (int j = 0; j < n; ++j) {
     const int st_v = wt.kv % NS;
@@ -354,21 +411,30 @@ __device__ __forceinline__ void mma_flash_pair(const Ctx& cx, Waits& wt, const b
       mbar_wait(&mi.kv_full[st_k], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
       ++wt.kv;
     }
-#pragma unroll
-    for (int b = 0; b < 2; ++b) {
-      if (!has[b] || j >= nb[b]) continue;
+    if (has_b && j < nb_b) {
+      // first half of P V as soon as keys 0..63 of P are in TMEM (no token: it is not on the
+      // other block's critical path for long, and the pipe is in order)
+      mbar_wait(&mi.p_half[b], full_par(wt.p[b]), cx.abort_flag, cx.status, W_PHALF);
+      tc_fence_after_sync();
+      issue_pv<D>(tO, tS, ring_u32 + st_v * C::TILE_BYTES, j > 0, 0, TILE / 32);
       mbar_wait(&mi.p_full[b], full_par(wt.p[b]), cx.abort_flag, cx.status, W_PFULL);
       ++wt.p[b];
+      turn_take(cx, wt, b);
       tc_fence_after_sync();
-      issue_pv<D>(tO[b], tS[b], ring_u32 + st_v * C::TILE_BYTES, j > 0);
-      if (j == nb[b] - 1) mma_commit(&mi.o_full[b]);
-      if (j + 1 < nb[b]) { issue_qk<D>(tS[b], q_u32[b], ring_u32 + st_k * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
+      issue_pv<D>(tO, tS, ring_u32 + st_v * C::TILE_BYTES, true, TILE / 32, TILE / 16);
+      if (j == nb_b - 1) mma_commit(&mi.o_full[b]);
+      if (j + 1 < nb_b) { issue_qk<D>(tS, q_u32, ring_u32 + st_k * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
+      turn_pass(cx, wt, b);
+      mma_commit(&mi.kv_free[st_v]);
+      if (more) mma_commit(&mi.kv_free[st_k]);
+    } else {                                   // stages this block never reads
+      turn_take(cx, wt, b);
+      turn_pass(cx, wt, b);
+      mbar_arrive(&mi.kv_free[st_v]);
+      if (more) mbar_arrive(&mi.kv_free[st_k]);
     }
-    mma_commit(&mi.kv_free[st_v]);
-    if (more) mma_commit(&mi.kv_free[st_k]);
   }
-#pragma unroll
-  for (int b = 0; b < 2; ++b) if (has[b]) ++wt.acc[b];
+  if (has_b) ++wt.acc[b];
 }
 
 // softmax group: online softmax over n key tiles for this thread's row; vis(j) = visible
@@ -384,7 +450,7 @@ __device__ __forceinline__ void wg_flash_loop(const Ctx& cx, uint32_t& n_s, uint
     mbar_wait(&mi.s_full[b], full_par(n_s), cx.abort_flag, cx.status, W_SFULL);
     ++n_s;
     tc_fence_after_sync();
-    softmax_tile<D>(tS, tO, vis(j), j == 0, scale_log2, m_used, l_run);
+    softmax_tile<D>(tS, tO, vis(j), j == 0, scale_log2, m_used, l_run, &mi.p_half[b]);
     tc_fence_before_sync();
     mbar_arrive(&mi.p_full[b]);
   }
@@ -427,6 +493,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   cx.tmem = mi.tmem_base;
+#if PC_SETMAXNREG
+  if (warp >= 8) setmaxnreg_dec<REGS_SERVICE>(); else setmaxnreg_inc<REGS_SOFTMAX>();
+#endif
 
   Waits wt;
 
@@ -484,11 +553,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       producer_drain(cx, wt);
     }
     __syncwarp();
-  } else if (warp == WARP_MMA) {
-    // ================================================================ tcgen05 issuer
+  } else if (warp == WARP_MMA || warp == WARP_MMA + 1) {
+    // ================================================================ tcgen05 issuers (one per block)
     if (lane == 0) {
+      const int b = warp - WARP_MMA;
       const uint32_t ring_u32 = smem_u32(cx.ring);
-      const uint32_t q_u32[2] = {smem_u32(cx.sQ[0]), smem_u32(cx.sQ[1])};
+      const uint32_t q_u32 = smem_u32(cx.sQ[b]);
       while (true) {
         const int item = consumer_next_item(cx, wt);
         if (item == ITEM_DONE) break;
@@ -497,34 +567,35 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int nsub = n_subitems(sch, within);
         for (int sub = 0; sub < nsub; ++sub) {
           const SubItem it = decode_sub(sch, hkv, within, sub);
-          const bool has[2] = {true, it.hB >= 0};
-          const int nb[2] = {it.tA + 1, it.hB >= 0 ? it.tB + 1 : 0};
-          mma_flash_pair<D>(cx, wt, has, nb);
+          const bool has_b = (b == 0) || it.hB >= 0;
+          const int nb_b = (b == 0) ? it.tA + 1 : (it.hB >= 0 ? it.tB + 1 : 0);
+          const int n = (it.hB >= 0 ? it.tB : it.tA) + 1;
+          mma_flash_block<D>(cx, wt, b, has_b, nb_b, n);
         }
         if (within == 0) {
-#pragma unroll
-          for (int b = 0; b < 2; ++b) mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
+          // ---- score sweep: this issuer computes the columns of its own block (window rows b*128..)
+          mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
           for (int u = 0; u < n_pass; ++u) {
             const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
             const int rows_total = heads * prm.w;
-            const int rows[2] = {rows_total < TILE ? rows_total : TILE, rows_total > TILE ? rows_total - TILE : 0};
-#pragma unroll
-            for (int b = 0; b < 2; ++b)
-              if (rows[b] > 0) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
+            const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
+            if (rows_b > 0) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
             for (int j = 0; j < sch.T; ++j) {
               const int e = j & 1;
-              mbar_wait(&mi.t_free[e], free_par(e ? wt.t[1] : wt.t[0]), cx.abort_flag, cx.status, W_TFREE);
+              mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
               const int st = wt.kv % NS;
               mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
               ++wt.kv;
-              tc_fence_after_sync();
-#pragma unroll
-              for (int b = 0; b < 2; ++b)
-                if (rows[b] > 0)
-                  issue_kq<D>(cx.tmem + e * 256 + b * 128, ring_u32 + st * C::TILE_BYTES, q_u32[b], (rows[b] + 15) & ~15);
-              mma_commit(&mi.t_full[e]);
-              mma_commit(&mi.kv_free[st]);
-              if (e) ++wt.t[1]; else ++wt.t[0];
+              if (rows_b > 0) {
+                tc_fence_after_sync();
+                issue_kq<D>(cx.tmem + e * 256 + b * 128, ring_u32 + st * C::TILE_BYTES, q_u32, (rows_b + 15) & ~15);
+                mma_commit(&mi.t_full[e]);
+                mma_commit(&mi.kv_free[st]);
+              } else {
+                mbar_arrive(&mi.t_full[e]);
+                mbar_arrive(&mi.kv_free[st]);
+              }
+              ++wt.t[e];
             }
           }
         }
@@ -700,6 +771,9 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
   __syncthreads();
   tc_fence_after_sync();
   cx.tmem = mi.tmem_base;
+#if PC_SETMAXNREG
+  if (warp >= 8) setmaxnreg_dec<REGS_SERVICE>(); else setmaxnreg_inc<REGS_SOFTMAX>();
+#endif
 
   Waits wt;
 
@@ -756,15 +830,15 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
       producer_drain(cx, wt);
     }
     __syncwarp();
-  } else if (warp == WARP_MMA) {
+  } else if (warp == WARP_MMA || warp == WARP_MMA + 1) {
     if (lane == 0) {
+      const int b = warp - WARP_MMA;
       while (true) {
         const int item = consumer_next_item(cx, wt);
         if (item == ITEM_DONE) break;
         const Dec d = decode(item);
-        const bool has[2] = {d.rows[0] > 0, d.rows[1] > 0};
-        const int nb[2] = {has[0] ? d.n : 0, has[1] ? d.n : 0};
-        mma_flash_pair<D>(cx, wt, has, nb);
+        const bool has_b = d.rows[b] > 0;
+        mma_flash_block<D>(cx, wt, b, has_b, has_b ? d.n : 0, d.n);
       }
     }
     __syncwarp();
