@@ -11,6 +11,7 @@ struct PrefillParams {
   int C, L, w, Hq, Hkv;
   float scale_log2;              // softmax scale * log2(e)
   const double2* rope_tab;       // [L][d/2] (cos, sin)
+  const float4* rope_tab32;      // [L][d/2] (cos_hi, cos_lo, sin_hi, sin_lo): fp32 split of the same values (head size 128)
   float* lse;                    // [C,Hq,L] or null
   float* win_lse;                // [C,Hq,w]
   float* win_score;              // [C,Hkv,L]
@@ -20,6 +21,9 @@ struct PrefillParams {
 
 // maps: q (box 64x1x128x1), k_rot, v, o (store), q with a w-row box
 cudaError_t launch_prefill_attn(const CUtensorMap* maps, const PrefillParams& prm, int d, int grid, cudaStream_t st);
+
+// Head size 128: CTA-pair kernel (pc_prefill2.cu).  maps as above plus maps[5] = rotated keys with a 64-token box.
+cudaError_t launch_prefill_pair(const CUtensorMap* maps, const PrefillParams& prm, int sm_count, cudaStream_t st);
 
 struct ParallelParams {
   int B, w, Hq, Hkv, Nk;
