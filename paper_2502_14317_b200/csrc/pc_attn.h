@@ -11,7 +11,6 @@ struct PrefillParams {
   int C, L, w, Hq, Hkv;
   float scale_log2;              // softmax scale * log2(e)
   const double2* rope_tab;       // [L][d/2] (cos, sin)
-  const float4* rope_tab32;      // [L][d/2] (cos_hi, cos_lo, sin_hi, sin_lo): fp32 split of the same values (head size 128)
   float* lse;                    // [C,Hq,L] or null
   float* win_lse;                // [C,Hq,w]
   float* win_score;              // [C,Hkv,L]

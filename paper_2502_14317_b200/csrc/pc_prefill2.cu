@@ -31,9 +31,6 @@
 #ifndef PC2_EARLY_ROT
 #define PC2_EARLY_ROT 1
 #endif
-#ifndef PC2_ROPE_FP32
-#define PC2_ROPE_FP32 1
-#endif
 #ifndef PC2_POLY_PAIRS_PER_8
 #define PC2_POLY_PAIRS_PER_8 2
 #endif
@@ -172,74 +169,35 @@ __device__ __forceinline__ void mbar_wait_cluster(uint64_t* bar, uint32_t parity
   }
 }
 
-// RoPE of a Q tile in shared memory.  The rotation is evaluated in fp32 with the fp64 table value
-// split into hi + lo parts; the result carries an error below 2^-23 (|x1| + |x2|), and only when it
-// falls that close to a bf16 rounding boundary (about one pair in 10^4) is the pair recomputed in
-// fp64, so the rounded values are those of the fp64 evaluation.  fp64 arithmetic runs at a small
-// fraction of the fp32 rate on this GPU: doing every element in fp64 costs a tenth of the kernel.
-// RoPE of 8 pairs of row `row` of a 128-byte-swizzled [128 x 128] bf16 tile (two atoms of 64
-// columns): pairs (t, t + 64) for t in [8 * cidx, 8 * cidx + 8).  tab32: (cos_hi, cos_lo, sin_hi,
-// sin_lo) per pair; tab64: (cos, sin) in fp64 for the rare exact path.
-struct RopeEntries { float4 v[8]; };
-__device__ __forceinline__ void rope_load_entries(RopeEntries& e, const float4* __restrict__ tab32, int cidx) {
+// RoPE of half of row `row` of a 128-byte-swizzled [128 x 128] bf16 Q tile (two atoms of 64 columns):
+// pairs (t, t + 64) for t in [32 * part, 32 * part + 32) at position `pos`; fp64, one rounding.
+__device__ __forceinline__ void rope_row_part(uint8_t* tile, int row, int part, int pos, const double2* __restrict__ tab) {
+  const double2* tab_row = tab + (size_t)pos * (D / 2);
+#pragma unroll 2
+  for (int cidx = part * 4; cidx < part * 4 + 4; ++cidx) {
+    uint8_t* lo_p = tile + sw128_offset(row, cidx);
+    uint8_t* hi_p = tile + 16384 + sw128_offset(row, cidx);
+    const uint4 lo = *reinterpret_cast<const uint4*>(lo_p);
+    const uint4 hi = *reinterpret_cast<const uint4*>(hi_p);
+    const uint32_t lo_w[4] = {lo.x, lo.y, lo.z, lo.w}, hi_w[4] = {hi.x, hi.y, hi.z, hi.w};
+    uint32_t out_lo[4], out_hi[4];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) e.v[i] = __ldg(tab32 + cidx * 8 + i);
-}
-__device__ __forceinline__ void rope_chunk_pair(uint8_t* tile, int row, int cidx, const RopeEntries& ent,
-                                                const double2* __restrict__ tab64) {
-  uint8_t* lo_p = tile + sw128_offset(row, cidx);
-  uint8_t* hi_p = tile + 16384 + sw128_offset(row, cidx);
-  const uint4 lo = *reinterpret_cast<const uint4*>(lo_p);
-  const uint4 hi = *reinterpret_cast<const uint4*>(hi_p);
-  const uint32_t lo_w[4] = {lo.x, lo.y, lo.z, lo.w}, hi_w[4] = {hi.x, hi.y, hi.z, hi.w};
-  uint32_t out_lo[4], out_hi[4];
+    for (int i = 0; i < 4; ++i) {
+      uint32_t rl = 0, rh = 0;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint32_t rl = 0, rh = 0;
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const float x1 = __uint_as_float(((lo_w[i] >> (16 * e)) & 0xFFFFu) << 16);
-      const float x2 = __uint_as_float(((hi_w[i] >> (16 * e)) & 0xFFFFu) << 16);
-      const float4 cs = ent.v[2 * i + e];
-#if !PC2_ROPE_FP32
-      {
-        const double2 cd = tab64[cidx * 8 + 2 * i + e];
-        rl |= (uint32_t)f64_to_bf16_rne((double)x1 * cd.x - (double)x2 * cd.y) << (16 * e);
-        rh |= (uint32_t)f64_to_bf16_rne((double)x2 * cd.x + (double)x1 * cd.y) << (16 * e);
-        continue;
+      for (int e = 0; e < 2; ++e) {
+        const double x1 = (double)__uint_as_float(((lo_w[i] >> (16 * e)) & 0xFFFFu) << 16);
+        const double x2 = (double)__uint_as_float(((hi_w[i] >> (16 * e)) & 0xFFFFu) << 16);
+        const double2 t = tab_row[cidx * 8 + 2 * i + e];
+        rl |= (uint32_t)f64_to_bf16_rne(x1 * t.x - x2 * t.y) << (16 * e);
+        rh |= (uint32_t)f64_to_bf16_rne(x2 * t.x + x1 * t.y) << (16 * e);
       }
-#endif
-      const float tl = fmaf(x1, cs.y, -x2 * cs.w), rlo = fmaf(x1, cs.x, fmaf(-x2, cs.z, tl));
-      const float th = fmaf(x2, cs.y, x1 * cs.w), rhi = fmaf(x2, cs.x, fmaf(x1, cs.z, th));
-      const float tol = 4.76837158e-7f * (fabsf(x1) + fabsf(x2));          // 2^-21: four times the fp32 error bound
-      const uint32_t bl = __float_as_uint(rlo), bh = __float_as_uint(rhi);
-      const float midl = __uint_as_float((bl & 0xFFFF0000u) | 0x8000u), midh = __uint_as_float((bh & 0xFFFF0000u) | 0x8000u);
-      uint32_t vl = (bl + 0x7FFFu + ((bl >> 16) & 1u)) >> 16, vh = (bh + 0x7FFFu + ((bh >> 16) & 1u)) >> 16;
-      if (fabsf(rlo - midl) <= tol || fabsf(rhi - midh) <= tol) {          // too close to a bf16 rounding boundary
-        const double2 cd = tab64[cidx * 8 + 2 * i + e];
-        vl = f64_to_bf16_rne((double)x1 * cd.x - (double)x2 * cd.y);
-        vh = f64_to_bf16_rne((double)x2 * cd.x + (double)x1 * cd.y);
-      }
-      rl |= vl << (16 * e);
-      rh |= vh << (16 * e);
+      out_lo[i] = rl;
+      out_hi[i] = rh;
     }
-    out_lo[i] = rl;
-    out_hi[i] = rh;
+    *reinterpret_cast<uint4*>(lo_p) = make_uint4(out_lo[0], out_lo[1], out_lo[2], out_lo[3]);
+    *reinterpret_cast<uint4*>(hi_p) = make_uint4(out_hi[0], out_hi[1], out_hi[2], out_hi[3]);
   }
-  *reinterpret_cast<uint4*>(lo_p) = make_uint4(out_lo[0], out_lo[1], out_lo[2], out_lo[3]);
-  *reinterpret_cast<uint4*>(hi_p) = make_uint4(out_hi[0], out_hi[1], out_hi[2], out_hi[3]);
-}
-
-// Rotate half of row `row` (chunk pairs 4 * part .. 4 * part + 3) at RoPE position `pos`.
-__device__ __forceinline__ void rope_row_part(uint8_t* tile, int row, int part, int pos, const float4* __restrict__ tab32,
-                                              const double2* __restrict__ tab64) {
-  const float4* t32 = tab32 + (size_t)pos * (D / 2);
-  const double2* t64 = tab64 + (size_t)pos * (D / 2);
-  RopeEntries e[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) rope_load_entries(e[i], t32, part * 4 + i);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) rope_chunk_pair(tile, row, part * 4 + i, e[i], t64);
 }
 
 __device__ __forceinline__ void init_barriers2(Misc2& mi) {
@@ -523,7 +481,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int tok = b.t * TILE + r;
       WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
       ++cQ;
-      if (tok < prm.L) rope_row_part(cx.sQ[qb], r, hlf, tok, prm.rope_tab32, prm.rope_tab);
+      if (tok < prm.L) rope_row_part(cx.sQ[qb], r, hlf, tok, prm.rope_tab);
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.q_ready[qb], 0));
@@ -744,7 +702,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int qb = cQ & 1;
           WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
           ++cQ;
-          if (r < rows_half) rope_row_part(cx.sQ[qb], r, hlf, prm.L - prm.w + (r % prm.w), prm.rope_tab32, prm.rope_tab);
+          if (r < rows_half) rope_row_part(cx.sQ[qb], r, hlf, prm.L - prm.w + (r % prm.w), prm.rope_tab);
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.q_ready[qb], 0));

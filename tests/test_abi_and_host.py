@@ -45,11 +45,11 @@ def test_status_strings_and_version(lib):
 
 def test_workspace_queries_are_host_only(lib):
     from paper_2502_14317_b200 import binding
-    # cfg1: 256 B counter + fp64 cos/sin table L * d/2 * 16 B + its fp32 hi/lo copy (head size 128)
-    assert binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128) == 256 + 2 * 8192 * 64 * 16
+    # cfg1: 256 B counter + fp64 cos/sin table L * d/2 * 16 B
+    assert binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128) == 256 + 8192 * 64 * 16
     assert binding.chunk_prefill_attn_workspace_bytes(4, 256, 16, 4, 2, 64) == 256 + 256 * 32 * 16
     with_krot = binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128, k_rot_in_workspace=True)
-    assert with_krot == 256 + 2 * 8192 * 64 * 16 + 16 * 8192 * 8 * 128 * 2
+    assert with_krot == 256 + 8192 * 64 * 16 + 16 * 8192 * 8 * 128 * 2
     # unsupported shapes give 0
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 24, 4, 2, 64) == 0       # window not a power of two
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 2, 96) == 0       # head size

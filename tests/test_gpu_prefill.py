@@ -47,6 +47,13 @@ def test_cfg0_full(cfg0_inputs):
     (1, 100, 32, 8, 1, 64, 10000.0),       # single ragged tile, G*w = 256 window rows
     (1, 640, 64, 8, 1, 128, 500000.0),     # G*w = 512 window rows: two score passes
     (1, 130, 64, 1, 1, 64, 10000.0),       # single head, MHA, two tiles with a 2-token tail
+    # head size 128 runs on CTA pairs: two q-heads (or two adjacent query tiles) per pair
+    (2, 300, 16, 2, 1, 128, 10000.0),      # G=2: one head pair, ragged last tile
+    (1, 100, 32, 1, 1, 128, 10000.0),      # MHA, a single ragged tile: the second CTA of the pair has no block
+    (1, 256, 128, 4, 2, 128, 500000.0),    # widest window = exactly the last tile, two kv-heads
+    (2, 1100, 64, 6, 2, 128, 10000.0),     # G=3 (odd): tile-pair mode, 9 tiles, ragged
+    (1, 1024, 8, 2, 2, 128, 10000.0),      # MHA, even tile count, smallest window
+    (1, 200, 128, 8, 1, 128, 10000.0),     # G*w = 1024 window rows: four score passes, window over two tiles
 ])
 def test_shapes(C, L, w, Hq, Hkv, d, theta):
     rng = np.random.default_rng(L * 7 + Hq)
@@ -55,6 +62,20 @@ def test_shapes(C, L, w, Hq, Hkv, d, theta):
     v = pc_inputs.f32_to_bf16_bits(rng.standard_normal((C, L, Hkv, d)).astype(np.float32))
     k[:, 0] = pc_inputs.f32_to_bf16_bits(pc_inputs.bf16_bits_to_f32(k[:, 0]) * np.float32(4.0))
     _run_and_compare(q, k, v, w, theta)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_growing_logits_rescale_path(d):
+    """Keys whose norm grows along the chunk make the running row maximum jump by more than the lazy
+    threshold again and again, so the accumulator is rescaled in most tiles (rare otherwise)."""
+    rng = np.random.default_rng(99 + d)
+    C, L, Hq, Hkv, w = 1, 700, 4, 2, 32
+    q = rng.standard_normal((C, L, Hq, d)).astype(np.float32)
+    k = rng.standard_normal((C, L, Hkv, d)).astype(np.float32)
+    v = rng.standard_normal((C, L, Hkv, d)).astype(np.float32)
+    k *= np.linspace(1.0, 40.0, L, dtype=np.float32)[None, :, None, None]
+    bits = [pc_inputs.f32_to_bf16_bits(x) for x in (q, k, v)]
+    _run_and_compare(bits[0], bits[1], bits[2], w, 10000.0)
 
 
 def test_deterministic_and_strided(cfg0_inputs):
@@ -72,6 +93,20 @@ def test_deterministic_and_strided(cfg0_inputs):
     for key in ("o", "k_rot", "win_score", "win_lse"):
         assert torch.equal(a[key], b[key]), f"{key} not reproducible run to run"
         assert torch.equal(a[key], c[key]), f"{key} differs for strided inputs"
+
+
+def test_deterministic_head_size_128():
+    """The CTA-pair kernel (two issuing threads, two softmax warpgroups on alternate tiles) must give the same
+    bits run to run: accumulation order and score sums are fixed by construction."""
+    import paper_2502_14317_b200 as pc
+    rng = np.random.default_rng(5)
+    q = to_dev(pc_inputs.f32_to_bf16_bits(rng.standard_normal((2, 900, 8, 128)).astype(np.float32)))
+    k = to_dev(pc_inputs.f32_to_bf16_bits(rng.standard_normal((2, 900, 2, 128)).astype(np.float32)))
+    v = to_dev(pc_inputs.f32_to_bf16_bits(rng.standard_normal((2, 900, 2, 128)).astype(np.float32)))
+    runs = [pc.chunk_prefill_attn(q, k, v, w=64, rope_theta=5e5, want_lse=True) for _ in range(3)]
+    torch.cuda.synchronize()
+    for key in ("o", "win_score", "win_lse", "lse"):
+        assert torch.equal(runs[0][key], runs[1][key]) and torch.equal(runs[0][key], runs[2][key]), key
 
 
 def test_argument_errors():
