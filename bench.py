@@ -293,6 +293,12 @@ def run_gpu(args, cfg):
     value = replica_throughput(tokens, world, ms_per_step)
 
     if rank == 0:
+        # DRAM bytes per launch of the dominant kernel, from the ncu capture summarised in
+        # profiles/prefill_pair_kernel_cfg1_C2_ncu_full.md (2 of 16 chunks captured, scaled by the chunk count)
+        traffic, traffic_note = args.traffic_bytes, "command line"
+        if traffic is None and args.workload == "cfg1":
+            traffic = 350.46e6 / 2 * cfg.C
+            traffic_note = "ncu dram__bytes_read+write of a 2-chunk launch (350.46 MB) scaled to %d chunks" % cfg.C
         flops = prefill_flops(cfg)
         ach_tflops = flops / (stage_ms["prefill_attn"] * 1e-3) / 1e12
         gather_bytes = 2.0 * (2 * cfg.Hkv * cfg.m * cfg.k * cfg.d * 2)
@@ -308,14 +314,14 @@ def run_gpu(args, cfg):
                     "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
                     "d2h_bytes_per_step": int(h_out.numel()) * 2, "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": {"bound": "tensor", "kernel": "prefill_attn_kernel (+ RoPE pre-pass inside the same call)",
+            "roofline": {"bound": "tensor", "kernel": "prefill_pair_kernel (+ RoPE table and key pre-pass inside the same call)",
                          "achieved": ach_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                          "frac": ach_tflops / peaks["bf16_tflops_sustained"],
                          "frac_of_burst_peak": ach_tflops / peaks["bf16_tflops"],
                          "frac_of_nominal_2250": ach_tflops / 2250.0,
                          "peak_source": peaks["source"] + " cuBLAS bf16, sustained (kernel timed inside a long step)",
                          "algorithmic_flops_per_launch": flops, "ms_per_launch": stage_ms["prefill_attn"],
-                         "traffic": args.traffic_bytes},
+                         "traffic": traffic, "traffic_note": traffic_note},
             "stages": {
                 "prefill_attn": {"ms": stage_ms["prefill_attn"], "tflops": ach_tflops},
                 "score_select": {"ms": stage_ms["score_select"], "algorithmic_bytes": sel_bytes,
@@ -328,6 +334,8 @@ def run_gpu(args, cfg):
                                   "tflops": par_flops / (stage_ms["parallel_attn"] * 1e-3) / 1e12},
             },
         }
+        if world == 1 and not args.no_extra:
+            line["extra"] = extra_measurements(pc, torch, dev, peaks)
         if not args.no_cpu_baseline and world == 1:
             v_cpu, s_cpu, desc = oracle_sample(cfg)
             line["cpu_baseline"] = {"value": v_cpu, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
@@ -338,6 +346,75 @@ def run_gpu(args, cfg):
         dist.destroy_process_group()
 
 
+def _time_us(torch, fn, warm=3, reps=20):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return 1e3 * e0.elapsed_time(e1) / reps
+
+
+def extra_measurements(pc, torch, dev, peaks) -> dict:
+    """Single-call timings of the stages whose full-size workloads are not part of the cfg1 step
+    (outside the timed region; random device data, parity is covered by the tests):
+    parallel attention over a batch of compressed caches (cfg4), token top-k on enough rows to be
+    bandwidth-bound, and the gather at the cfg2 size."""
+    out = {}
+    g = torch.Generator(device=dev).manual_seed(4)
+    # ---- cfg4: B=64 sequences x (8 kept chunks x 2048 keys), 64 window queries
+    B, w, Hq, Hkv, d, Nk = 64, 64, 32, 8, 128, 16384
+    qw = torch.randn((B, w, Hq, d), device=dev, generator=g).bfloat16()
+    kc = torch.randn((B, Hkv, Nk, d), device=dev, generator=g).bfloat16()
+    vc = torch.randn((B, Hkv, Nk, d), device=dev, generator=g).bfloat16()
+    kw = torch.randn((B, w, Hkv, d), device=dev, generator=g).bfloat16()
+    vw = torch.randn((B, w, Hkv, d), device=dev, generator=g).bfloat16()
+    buf = {}
+
+    def run_par():
+        r = pc.parallel_attn(qw, kc, vc, kw, vw, q_pos0=8128, rope_theta=5e5, out=buf.get("out"), status=buf.get("status"),
+                             workspace=buf.get("workspace"))
+        buf.update(r)
+    us = _time_us(torch, run_par, reps=10)
+    flops = 4.0 * d * (Nk + (w + 1) / 2) * w * Hq * B
+    kv_bytes = 2.0 * B * Hkv * Nk * d * 2
+    out["parallel_attn_cfg4"] = {"us": us, "tflops": flops / us / 1e6, "kv_gbs": kv_bytes / us / 1e3,
+                                 "frac_of_measured_bf16_burst": flops / us / 1e6 / peaks["bf16_tflops"],
+                                 "frac_of_measured_hbm": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
+                                 "flops": flops, "kv_bytes": kv_bytes, "l2": "4.3 GB of K/V per call, larger than L2"}
+    del qw, kc, vc, kw, vw, buf
+    # ---- token top-k, cfg1 row shape (8128 candidates -> 2048) on 65536 rows (2.1 GB of scores)
+    C, Hk, L, n_cand, k = 8192, 8, 8192, 8128, 2048
+    score = torch.rand((C, Hk, L), device=dev, generator=g)
+    kept = torch.arange(C, device=dev, dtype=torch.int32)
+    idx = torch.empty((C, Hk, k), device=dev, dtype=torch.int32)
+    us = _time_us(torch, lambda: pc.select_tokens(score, kept, n_cand, k, out=idx), reps=5)
+    sel_bytes = 4.0 * C * Hk * (n_cand + k)
+    out["select_tokens_65536_rows"] = {"us": us, "algorithmic_bytes": sel_bytes, "gbs": sel_bytes / us / 1e3,
+                                       "frac_of_measured_hbm": sel_bytes / us / 1e3 / peaks["hbm_gbs"]}
+    del score, idx
+    # ---- gather at the cfg2 size: 12 kept chunks x 1024 tokens x 32 heads (201 MB read + 201 MB written)
+    C2, L2, H2, m2, k2 = 32, 4096, 32, 12, 1024
+    ksrc = torch.randn((C2, L2, H2, d), device=dev, generator=g).bfloat16()
+    vsrc = torch.randn((C2, L2, H2, d), device=dev, generator=g).bfloat16()
+    kept2 = torch.arange(0, 2 * m2, 2, device=dev, dtype=torch.int32)
+    idx2 = torch.sort(torch.rand((m2, H2, L2 - 64), device=dev, generator=g).argsort(-1)[..., :k2], -1).values.to(torch.int32)
+    gb = {}
+
+    def run_gather():
+        gb["k"], gb["v"], gb["p"] = pc.gather_kv(ksrc, vsrc, kept2, idx2, k_out=gb.get("k"), v_out=gb.get("v"), pos_out=gb.get("p"))
+    us = _time_us(torch, run_gather, reps=20)
+    g_bytes = 2.0 * (2 * H2 * m2 * k2 * d * 2)
+    out["gather_cfg2"] = {"us": us, "algorithmic_bytes": g_bytes, "gbs": g_bytes / us / 1e3,
+                          "frac_of_measured_hbm": g_bytes / us / 1e3 / peaks["hbm_gbs"],
+                          "l2": "sources 2 x 1.07 GB, larger than L2"}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -346,6 +423,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the single-call timings of cfg4 / scaled select / cfg2 gather")
     ap.add_argument("--chunks", type=int, default=None,
                     help="override the number of chunks (smaller case of the same workload, e.g. for an ncu capture)")
     ap.add_argument("--traffic-bytes", type=float, default=None,

@@ -64,111 +64,149 @@ void launch_select_chunks(const float* score, int C, int m, int lower_is_better,
 }
 
 // ------------------------------------------------------------------ token top-k
-// One CTA per (kept chunk, kv-head) row.  The row's keys sit in shared memory; an
-// 8-bit-digit radix search finds the k-th largest key T, then one ordered sweep emits
-// the positions with key > T plus the first (k - count_gt) positions with key == T,
-// so ties go to the lower position and the output is ascending.
-constexpr int SEL_THREADS = 1024;
-constexpr int SEL_WARPS = SEL_THREADS / 32;
+// One CTA per (kept chunk, kv-head) row, 32 candidates per thread held in REGISTERS.
+//   1. The row is read once with coalesced 16-byte loads into shared memory (padded by one
+//      word per 32 so that the next step is free of bank conflicts); every thread then takes
+//      the 32 consecutive positions [32 tid, 32 tid + 32) as order-preserving uint32 keys and
+//      transposes its 32 x 32 bit matrix in registers: word b then holds bit b of all 32 keys.
+//   2. The k-th largest key T is found bit by bit, most significant first.  On the bit slices a
+//      round is three instructions per thread (and, popc, add) plus one redux per warp, one
+//      shared-memory atomic per warp and one barrier: 32 rounds whatever the distribution of
+//      the scores, no histogram hot spots, and the masks of the keys > T and == T fall out.
+//   3. One block scan of (count > T, count == T) gives every thread its output offset; positions
+//      with key > T plus the first (k - count_gt) positions with key == T are staged in shared
+//      memory in ascending order (ties go to the lower position) and written out coalesced.
+// HBM traffic: the row once (4 B per candidate) + 4 B per kept index.
+constexpr int SEL_KPT = 32;                                    // keys per thread
+constexpr int SEL_MAX_THREADS = 1024;                          // n_cand <= 32768
 
-__global__ void __launch_bounds__(SEL_THREADS) select_tokens_kernel(const float* __restrict__ win_score,
-                                                                    const int* __restrict__ kept, int Hkv, int L,
-                                                                    int n_cand, int k, int* __restrict__ idx) {
-  extern __shared__ uint32_t sel_smem[];
-  uint32_t* keys = sel_smem;                                   // [n_cand]
-  uint32_t* hist = sel_smem + ((n_cand + 31) & ~31);           // [SEL_WARPS][256]
-  __shared__ uint32_t tot[256];
-  __shared__ uint32_t s_prefix, s_remaining;
-  __shared__ int2 scan[SEL_THREADS];
+__device__ __forceinline__ int sel_pad(int p) { return p + (p >> 5); }
 
-  const int row = blockIdx.x;                 // r * Hkv + hkv
+__global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const float* __restrict__ win_score,
+                                                                        const int* __restrict__ kept, int Hkv, int L,
+                                                                        int n_cand, int k, int* __restrict__ idx) {
+  extern __shared__ uint32_t sel_smem[];                       // [n_pad] keys, later reused for the staged output
+  __shared__ int s_cnt[32];                                    // per bit: keys of the row >= the candidate threshold
+  __shared__ int2 s_scan[32];
+
+  const int row = blockIdx.x;                                  // r * Hkv + hkv
   const int r = row / Hkv, hk = row % Hkv;
-  const int c = kept[r];
-  const float* src = win_score + ((size_t)c * Hkv + hk) * L;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   int* out = idx + (size_t)row * k;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  if (k >= n_cand) {                          // nothing to evict: identity, then -1 padding
-    for (int j = tid; j < k; j += SEL_THREADS) out[j] = j < n_cand ? j : -1;
+  if (tid < 32) s_cnt[tid] = 0;                                // visible after the barrier that follows the row load
+  if (k >= n_cand) {                                           // nothing to evict: identity, then -1 padding
+    for (int j = tid; j < k; j += blockDim.x) out[j] = j < n_cand ? j : -1;
     return;
   }
-  for (int j = tid; j < n_cand; j += SEL_THREADS) keys[j] = rank_key(src[j], false);
-  if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; }
-  __syncthreads();
+  const int c = kept[r];
+  const float* src = win_score + ((size_t)c * Hkv + hk) * L;
 
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int b = tid; b < SEL_WARPS * 256; b += SEL_THREADS) hist[b] = 0u;
-    __syncthreads();
-    const uint32_t prefix = s_prefix;
-    const uint32_t himask = shift == 24 ? 0u : (0xFFFFFFFFu << (shift + 8));
-    uint32_t* myhist = hist + warp * 256;
-    const int n_round = (n_cand + SEL_THREADS - 1) / SEL_THREADS * SEL_THREADS;
-    for (int j = tid; j < n_round; j += SEL_THREADS) {
-      const bool active = j < n_cand && ((keys[j < n_cand ? j : 0] & himask) == prefix);
-      const uint32_t digit = active ? ((keys[j] >> shift) & 0xFFu) : 0x100u;
-      const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-      if (active && lane == (__ffs(peers) - 1)) myhist[digit] += __popc(peers);   // one writer per digit per warp
-      __syncwarp();
+  // ---- 1. row -> shared memory (coalesced), -> registers (32 consecutive positions per thread)
+  if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+    const float4* src4 = reinterpret_cast<const float4*>(src);
+    const int n4 = n_cand >> 2;
+    for (int i = tid; i < n4; i += blockDim.x) {
+      const float4 v = __ldg(src4 + i);
+      const int p = 4 * i;                                     // 4 consecutive positions never straddle a pad slot
+      uint32_t* d = sel_smem + sel_pad(p);
+      d[0] = rank_key(v.x, false); d[1] = rank_key(v.y, false); d[2] = rank_key(v.z, false); d[3] = rank_key(v.w, false);
     }
-    __syncthreads();
-    if (tid < 256) {
-      uint32_t s = 0;
-      for (int wv = 0; wv < SEL_WARPS; ++wv) s += hist[wv * 256 + tid];
-      tot[tid] = s;
-    }
-    __syncthreads();
-    if (tid == 0) {
-      uint32_t remaining = s_remaining, above = 0;
-      int b = 255;
-      for (; b > 0; --b) {
-        if (above + tot[b] >= remaining) break;
-        above += tot[b];
+    for (int p = (n4 << 2) + tid; p < n_cand; p += blockDim.x) sel_smem[sel_pad(p)] = rank_key(__ldg(src + p), false);
+  } else {
+    for (int p = tid; p < n_cand; p += blockDim.x) sel_smem[sel_pad(p)] = rank_key(__ldg(src + p), false);
+  }
+  __syncthreads();
+  uint32_t key[SEL_KPT];
+  const int p0 = tid * SEL_KPT;
+#pragma unroll
+  for (int i = 0; i < SEL_KPT; ++i) key[i] = (p0 + i < n_cand) ? sel_smem[p0 + i + tid] : 0u;   // pad(p0 + i) = p0 + i + tid; 0 ranks below every candidate
+
+  // in-register transpose of the 32 x 32 bit matrix: afterwards key[31 - b] holds bit b of every
+  // key, the key at position p0 + i sitting at bit 31 - i
+  {
+    uint32_t m = 0x0000FFFFu;
+#pragma unroll
+    for (int j = 16; j != 0; j >>= 1, m ^= (m << j)) {
+#pragma unroll
+      for (int q = 0; q < 32; q = (q + j + 1) & ~j) {
+        const uint32_t t = (key[q] ^ (key[q + j] >> j)) & m;
+        key[q] ^= t;
+        key[q + j] ^= (t << j);
       }
-      s_remaining = remaining - above;
-      s_prefix = prefix | ((uint32_t)b << shift);
     }
-    __syncthreads();
   }
-  const uint32_t T = s_prefix;
-  const int need_eq = (int)s_remaining;        // how many keys equal to T are taken (lowest positions first)
 
-  // ordered emission: contiguous segment per thread, block scan of (count_gt, count_eq)
-  const int seg = (n_cand + SEL_THREADS - 1) / SEL_THREADS;
-  const int j0 = tid * seg, j1 = min(j0 + seg, n_cand);
-  int gt = 0, eq = 0;
-  for (int j = j0; j < j1; ++j) { gt += keys[j] > T; eq += keys[j] == T; }
-  scan[tid] = make_int2(gt, eq);
-  __syncthreads();
-  for (int off = 1; off < SEL_THREADS; off <<= 1) {            // Hillis-Steele inclusive scan
-    int2 v = scan[tid];
-    if (tid >= off) { int2 u = scan[tid - off]; v.x += u.x; v.y += u.y; }
+  // ---- 2. k-th largest key, bit by bit.  active: keys equal to T on the bits decided so far;
+  // above: keys already known to be larger than T.
+  uint32_t active = 0xFFFFFFFFu, above = 0u, T = 0u;
+  int n_above = 0;
+#pragma unroll
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t ones = active & key[31 - bit];
+    int cnt = n_above + __popc(ones);                          // keys >= (T | 1 << bit)
+    cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+    if (lane == 0) atomicAdd(&s_cnt[bit], cnt);
     __syncthreads();
-    scan[tid] = v;
-    __syncthreads();
+    if (s_cnt[bit] >= k) {                                     // at least k keys are that large: the k-th largest has this bit
+      T |= 1u << bit;
+      active = ones;
+    } else {
+      above |= ones;
+      n_above += __popc(ones);
+      active &= ~key[31 - bit];
+    }
   }
-  int gt_before = scan[tid].x - gt, eq_before = scan[tid].y - eq;
-  for (int j = j0; j < j1; ++j) {
-    const uint32_t key = keys[j];
-    if (key > T) {
-      out[gt_before + min(eq_before, need_eq)] = j;
+  // active = keys == T (padding keys are 0 and can only tie with NaN keys, which sit at lower positions)
+
+  // ---- 3. ordered emission
+  const int gt = n_above, eq = __popc(active);
+  int sgt = gt, seq = eq;                                      // inclusive warp scan of both counts
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int a = __shfl_up_sync(0xFFFFFFFFu, sgt, off), b2 = __shfl_up_sync(0xFFFFFFFFu, seq, off);
+    if (lane >= off) { sgt += a; seq += b2; }
+  }
+  if (lane == 31) s_scan[warp] = make_int2(sgt, seq);
+  __syncthreads();                                             // also: every thread is done reading the keys from shared memory
+  int gt_before = sgt - gt, eq_before = seq - eq, gt_total = 0;
+  for (int wv = 0; wv < nwarps; ++wv) {
+    const int2 t = s_scan[wv];
+    if (wv < warp) { gt_before += t.x; eq_before += t.y; }
+    gt_total += t.x;
+  }
+  const int need_eq = k - gt_total;                            // keys equal to T that are taken (lowest positions first)
+  int* stage = reinterpret_cast<int*>(sel_smem);               // [k]
+#pragma unroll
+  for (int i = 0; i < SEL_KPT; ++i) {
+    const uint32_t sel_bit = 0x80000000u >> i;
+    if (above & sel_bit) {
+      stage[gt_before + min(eq_before, need_eq)] = p0 + i;
       ++gt_before;
-    } else if (key == T) {
-      if (eq_before < need_eq) out[gt_before + eq_before] = j;
+    } else if (active & sel_bit) {
+      if (eq_before < need_eq) stage[gt_before + eq_before] = p0 + i;
       ++eq_before;
     }
   }
+  __syncthreads();
+  for (int j = tid; j < k; j += blockDim.x) out[j] = stage[j];
 }
 
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
                                  int* idx, cudaStream_t st) {
-  const size_t smem = ((size_t)((n_cand + 31) & ~31) + SEL_WARPS * 256) * sizeof(uint32_t);
+  int threads = ((n_cand + SEL_KPT - 1) / SEL_KPT + 31) / 32 * 32;
+  if (threads < 32) threads = 32;
+  if (threads > SEL_MAX_THREADS) return cudaErrorInvalidValue;
+  const size_t words = (size_t)n_cand + (n_cand >> 5) + 1;
+  const size_t stage = k < n_cand ? (size_t)k : 0;             // k >= n_cand writes the identity directly
+  const size_t smem = (words > stage ? words : stage) * sizeof(uint32_t);
   static size_t configured = 0;
   if (smem > 48 * 1024 && smem > configured) {
     cudaError_t e = cudaFuncSetAttribute(select_tokens_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = smem;
   }
-  select_tokens_kernel<<<m * Hkv, SEL_THREADS, smem, st>>>(win_score, kept, Hkv, L, n_cand, k, idx);
+  select_tokens_kernel<<<m * Hkv, threads, smem, st>>>(win_score, kept, Hkv, L, n_cand, k, idx);
   return cudaGetLastError();
 }
 
