@@ -27,9 +27,6 @@
 #include "pc_attn.h"
 #include "pc_sm100.cuh"
 
-#ifndef PC_SETMAXNREG
-#define PC_SETMAXNREG 0
-#endif
 #ifndef PC_POLY_PAIRS_PER_8
 #define PC_POLY_PAIRS_PER_8 2
 #endif
@@ -39,8 +36,7 @@ namespace pc {
 namespace {
 
 constexpr int TILE = 128;
-constexpr int NUM_THREADS = 384;               // 3 warpgroups: softmax 0, softmax 1, {producer, issuer, 2 idle warps}
-constexpr int REGS_SOFTMAX = 224, REGS_SERVICE = 56;   // per-thread registers after re-partitioning (sum <= 64 K)
+constexpr int NUM_THREADS = 384;               // 3 warpgroups: softmax 0, softmax 1, {producer, two issuers, one idle warp}
 constexpr int WARP_PRODUCER = 8;
 constexpr int WARP_MMA = 9;                 // issuer of block 0; WARP_MMA + 1 issues block 1
 constexpr int NS = 4;                       // K/V ring stages
@@ -493,9 +489,6 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   cx.tmem = mi.tmem_base;
-#if PC_SETMAXNREG
-  if (warp >= 8) setmaxnreg_dec<REGS_SERVICE>(); else setmaxnreg_inc<REGS_SOFTMAX>();
-#endif
 
   Waits wt;
 
@@ -771,9 +764,6 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
   __syncthreads();
   tc_fence_after_sync();
   cx.tmem = mi.tmem_base;
-#if PC_SETMAXNREG
-  if (warp >= 8) setmaxnreg_dec<REGS_SERVICE>(); else setmaxnreg_inc<REGS_SOFTMAX>();
-#endif
 
   Waits wt;
 

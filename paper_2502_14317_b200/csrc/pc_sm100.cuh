@@ -312,12 +312,6 @@ __device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& y0, floa
   y1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
 }
 
-// Register re-partitioning between warpgroups (all four warps of a warpgroup execute it).
-template <int N>
-__device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N>
-__device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-
 // Round an fp64 value to bf16, ties to even, in one rounding (no fp32 detour).
 __device__ __forceinline__ uint16_t f64_to_bf16_rne(double x) {
   // fp64 -> fp32 with round-to-odd keeps enough information for a second, exact RNE step
