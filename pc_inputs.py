@@ -97,6 +97,13 @@ CONFIGS = {
     # 256K stress, aggressive eviction
     "cfg3": PrefillConfig("cfg3", C=32, L=8192, w=64, Hq=32, Hkv=8, d=128, rope_theta=5.0e5,
                           m=4, k=512, n_planted_chunks=2, n_planted_keys=32, seed=BASE_SEED + 3),
+    # the paper's own hyper-parameters (App. C) on the Llama-3 shape: query window = last 8 tokens, half of
+    # every chunk kept, 3 chunks kept; 32K context to keep the test short
+    "paper_w8": PrefillConfig("paper_w8", C=4, L=8192, w=8, Hq=32, Hkv=8, d=128, rope_theta=5.0e5,
+                              m=3, k=4092, n_planted_chunks=1, n_planted_keys=32, seed=BASE_SEED + 5),
+    # 6K position reuse under a 24K KV budget (the Llama-3.1 / Qwen2.5 setting): chunks of 6144, Nk = 4 x 6016
+    "reuse6k": PrefillConfig("reuse6k", C=6, L=6144, w=64, Hq=32, Hkv=8, d=128, rope_theta=5.0e5,
+                             m=4, k=6016, n_planted_chunks=1, n_planted_keys=32, seed=BASE_SEED + 6),
     # parallel attention only, batch of compressed caches
     "cfg4": ParallelAttnConfig("cfg4", B=64, Nk=16384, w=64, Hq=32, Hkv=8, d=128, rope_theta=5.0e5,
                                q_pos0=8128, seg=2048, seed=BASE_SEED + 4),

@@ -100,6 +100,16 @@ def test_cfg3_stress_256k():
     _check_prefill_workload("cfg3", n_row_samples=24, n_groups=1)
 
 
+def test_paper_hyperparameters_w8_half_kept():
+    """Second workload shape: the paper's own settings (window of 8 tokens, half of each chunk kept, 3 chunks kept)."""
+    _check_prefill_workload("paper_w8", n_row_samples=24, n_groups=1)
+
+
+def test_position_reuse_6k_budget_24k():
+    """Second workload shape: 6K chunks (48 key tiles, not a power of two) with a 24K compressed cache."""
+    _check_prefill_workload("reuse6k", n_row_samples=24, n_groups=1)
+
+
 def test_cfg4_batch_of_compressed_caches():
     import paper_2502_14317_b200 as pc
     cfg = pc_inputs.get_config("cfg4")
