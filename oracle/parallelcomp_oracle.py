@@ -222,6 +222,32 @@ def select_tokens(win_score: np.ndarray, kept: np.ndarray, n_cand: int, k: int) 
     return idx
 
 
+def select_tokens_calibrated(win_score: np.ndarray, kept: np.ndarray, n_cand: int, k: int, n_s: int, n_r: int,
+                             lam_s: float, lam_m: float, lam_r: float) -> np.ndarray:
+    """Eq. 8 (attention calibration) followed by Eq. 7: in every kept chunk and kv-head, first evict the
+    candidates whose cumulative score EXCEEDS the threshold of their region, then keep the k highest-scored
+    of the rest.  Regions (App. C): R_s = the first n_s candidate positions, R_r = the last n_r candidate
+    positions, R_m = the remaining ones; a threshold of +inf switches a region off (the paper evicts one
+    token type per layer range).  The comparison is taken on the float32 score against the float32
+    threshold.  Returns idx [m,Hkv,k] int32, ascending positions, padded with -1 where fewer than k survive.
+    """
+    S = np.asarray(win_score, dtype=np.float32)
+    _, Hkv, _ = S.shape
+    lam = np.empty(n_cand, dtype=np.float32)
+    lam[:] = np.float32(lam_m)
+    lam[max(0, n_cand - n_r):] = np.float32(lam_r)
+    lam[:min(n_s, n_cand)] = np.float32(lam_s)                  # the sink region wins where the two overlap
+    idx = np.full((len(kept), Hkv, k), -1, dtype=np.int32)
+    for r, c in enumerate(kept):
+        for hk in range(Hkv):
+            row = S[c, hk, :n_cand]
+            alive = np.flatnonzero(~(row > lam))                 # NaN is not "greater": it stays (and ranks worst)
+            order = alive[np.argsort(_rank_key_desc(row[alive]), kind="stable")]
+            kk = min(k, len(order))
+            idx[r, hk, :kk] = np.sort(order[:kk])
+    return idx
+
+
 def select_chunks_streaming(chunk_score: np.ndarray, m: int, batch: int) -> np.ndarray:
     """The paper's online fixed-size priority queue: chunks arrive in batches, the queue
     keeps the m lowest scores seen so far (ties -> lower id).  Must equal select_chunks."""

@@ -217,3 +217,42 @@ def test_cfg0_structure(cfg0_inputs, cfg0_oracle):
     # window replicated: every chunk carries the same window tokens
     assert np.array_equal(inp["q"][0, cfg.ctx:], inp["q"][3, cfg.ctx:])
     assert np.array_equal(out["k_rot"][0, cfg.ctx:], out["k_rot"][1, cfg.ctx:])
+
+
+def test_select_tokens_calibrated_pins():
+    """Eq. 8 + Eq. 7.  Pins: thresholds at +inf reduce to Eq. 7; a brute-force loop; hand-made rows with the
+    three regions; survivors fewer than k are padded with -1; NaN is never 'above the threshold'."""
+    rng = np.random.default_rng(21)
+    C, Hkv, L, w = 3, 2, 60, 4
+    S = rng.random((C, Hkv, L)).astype(np.float32)
+    kept = np.array([0, 2], dtype=np.int32)
+    inf = float("inf")
+    assert np.array_equal(orc.select_tokens_calibrated(S, kept, L - w, 9, 5, 7, inf, inf, inf),
+                          orc.select_tokens(S, kept, L - w, 9))
+    # brute force: per row, loop over positions, drop those above their region's threshold, take the k largest
+    n_cand, k, n_s, n_r, ls, lm, lr = L - w, 12, 5, 7, 0.5, 0.8, 0.3
+    got = orc.select_tokens_calibrated(S, kept, n_cand, k, n_s, n_r, ls, lm, lr)
+    for r, c in enumerate(kept):
+        for hk in range(Hkv):
+            alive = []
+            for j in range(n_cand):
+                lam = ls if j < n_s else (lr if j >= n_cand - n_r else lm)
+                if not (S[c, hk, j] > np.float32(lam)):
+                    alive.append(j)
+            best = sorted(alive, key=lambda j: (-float(S[c, hk, j]), j))[:k]
+            exp = sorted(best) + [-1] * (k - len(best))
+            assert got[r, hk].tolist() == exp
+    # hand-made row: positions 0..9, n_s = 2, n_r = 3 -> regions s = {0,1}, m = {2..6}, r = {7,8,9}
+    row = np.array([[[9.0, 0.1, 5.0, 0.2, 0.3, 6.0, 0.4, 7.0, 0.5, 0.6]]], dtype=np.float32)
+    one = np.array([0])
+    assert orc.select_tokens_calibrated(row, one, 10, 3, 2, 3, inf, inf, inf)[0, 0].tolist() == [0, 5, 7]
+    assert orc.select_tokens_calibrated(row, one, 10, 3, 2, 3, 1.0, inf, inf)[0, 0].tolist() == [2, 5, 7]     # sink evicted
+    assert orc.select_tokens_calibrated(row, one, 10, 3, 2, 3, inf, 5.5, inf)[0, 0].tolist() == [0, 2, 7]     # middle peak evicted
+    assert orc.select_tokens_calibrated(row, one, 10, 3, 2, 3, inf, inf, 0.55)[0, 0].tolist() == [0, 2, 5]    # recency peaks evicted
+    assert orc.select_tokens_calibrated(row, one, 10, 3, 2, 3, 0.0, 0.0, 0.0)[0, 0].tolist() == [-1, -1, -1]  # everything evicted
+    few = orc.select_tokens_calibrated(row, one, 10, 6, 2, 3, 0.05, 0.25, 0.45)[0, 0].tolist()
+    assert few == [3, -1, -1, -1, -1, -1]                                                                    # only 0.2 survives
+    # equality with the threshold is kept (strictly greater is evicted); NaN is kept and ranks last
+    row2 = np.array([[[0.5, np.nan, 0.7, 0.5]]], dtype=np.float32)
+    assert orc.select_tokens_calibrated(row2, one, 4, 4, 0, 0, inf, 0.5, inf)[0, 0].tolist() == [0, 1, 3, -1]
+    assert orc.select_tokens_calibrated(row2, one, 4, 2, 0, 0, inf, 0.5, inf)[0, 0].tolist() == [0, 3]
