@@ -126,6 +126,23 @@ PC_API int32_t pc_select_tokens(const float* win_score, const int32_t* kept, int
                          int32_t L, int32_t n_cand, int32_t k, int32_t* idx, void* stream);
 
 /* ------------------------------------------------------------------------------------
+ * Token eviction with attention calibration.  Paper: Sec. 3.1 "Attention calibration", Eq. 8,
+ * with the regions of App. C; combined here with the top-k of Eq. 7.
+ * For row (r, hkv): first evict every candidate j < n_cand whose score
+ * win_score[kept[r], hkv, j] EXCEEDS the threshold of its region - lambda_s for the first n_s
+ * positions (sink tokens, R_s), lambda_r for the last n_r candidate positions (recency
+ * tokens, R_r), lambda_m for the rest (R_m); +infinity switches a region off - then keep the
+ * k largest of the survivors as pc_select_tokens does (ties to the lower position, NaN is
+ * never above a threshold and ranks worst, ascending output).  Where fewer than k survive,
+ * the tail of idx[r,hkv,:] is -1 (pc_gather_kv turns those into zero rows).  The comparison
+ * is made on the fp32 score against the fp32 threshold.  Same limits as pc_select_tokens;
+ * n_s, n_r >= 0; where the first two regions overlap the sink region wins.
+ */
+PC_API int32_t pc_select_tokens_calibrated(const float* win_score, const int32_t* kept, int32_t C, int32_t m,
+                                    int32_t Hkv, int32_t L, int32_t n_cand, int32_t k, int32_t n_s, int32_t n_r,
+                                    float lambda_s, float lambda_m, float lambda_r, int32_t* idx, void* stream);
+
+/* ------------------------------------------------------------------------------------
  * Compressed cache.  Paper: Eq. 7 (K[R], V[R]) and Eq. 9 (concatenation over chunks).
  *     k_out[hkv, r*k + t, :] = k_src[kept[r], idx[r,hkv,t], hkv, :]     (same for v)
  *     pos_out[hkv, r*k + t]  = idx[r,hkv,t]

@@ -54,6 +54,8 @@ def load_library():
     lib.pc_select_chunks.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
     lib.pc_select_tokens.restype = c_int32
     lib.pc_select_tokens.argtypes = [c_void_p, c_void_p] + [c_int32] * 6 + [c_void_p, c_void_p]
+    lib.pc_select_tokens_calibrated.restype = c_int32
+    lib.pc_select_tokens_calibrated.argtypes = [c_void_p, c_void_p] + [c_int32] * 8 + [c_float] * 3 + [c_void_p, c_void_p]
     lib.pc_gather_kv.restype = c_int32
     lib.pc_gather_kv.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_int32, c_void_p, c_void_p] + [c_int32] * 4 + \
                                 [c_void_p, c_void_p, c_void_p, c_void_p]
@@ -181,6 +183,20 @@ def select_tokens(win_score, kept, n_cand, k, out=None):
     out = torch.empty((m, Hkv, k), dtype=torch.int32, device=win_score.device) if out is None else out
     _check(lib.pc_select_tokens(_ptr(win_score), _ptr(kept), C, m, Hkv, L, int(n_cand), int(k), _ptr(out), _stream()),
            "pc_select_tokens")
+    return out
+
+
+def select_tokens_calibrated(win_score, kept, n_cand, k, *, n_s=100, n_r=100, lambda_s=float("inf"),
+                             lambda_m=float("inf"), lambda_r=float("inf"), out=None):
+    """pc_select_tokens_calibrated: Eq. 8 eviction of over-attended tokens per region, then the top-k of Eq. 7."""
+    lib = load_library()
+    _need_cuda(win_score, kept)
+    C, Hkv, L = win_score.shape
+    m = kept.numel()
+    out = torch.empty((m, Hkv, k), dtype=torch.int32, device=win_score.device) if out is None else out
+    _check(lib.pc_select_tokens_calibrated(_ptr(win_score), _ptr(kept), C, m, Hkv, L, int(n_cand), int(k), int(n_s),
+                                           int(n_r), float(lambda_s), float(lambda_m), float(lambda_r), _ptr(out),
+                                           _stream()), "pc_select_tokens_calibrated")
     return out
 
 

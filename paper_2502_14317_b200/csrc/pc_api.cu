@@ -188,7 +188,24 @@ int32_t pc_select_tokens(const float* win_score, const int32_t* kept, int32_t C,
   if (C < 1 || m < 1 || m > C || Hkv < 1 || L < 1 || n_cand < 1 || n_cand > L || k < 1) return PC_ERR_INVALID_ARG;
   if (n_cand > 32768) return PC_ERR_UNSUPPORTED;
   if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
-  if (pc::launch_select_tokens(win_score, kept, m, Hkv, L, n_cand, k, idx, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+  if (pc::launch_select_tokens(win_score, kept, m, Hkv, L, n_cand, k, idx, nullptr, static_cast<cudaStream_t>(stream)) !=
+      cudaSuccess)
+    return PC_ERR_CUDA;
+  return PC_OK;
+}
+
+// ------------------------------------------------------------------------------------ token top-k with attention calibration
+int32_t pc_select_tokens_calibrated(const float* win_score, const int32_t* kept, int32_t C, int32_t m, int32_t Hkv,
+                                    int32_t L, int32_t n_cand, int32_t k, int32_t n_s, int32_t n_r, float lambda_s,
+                                    float lambda_m, float lambda_r, int32_t* idx, void* stream) {
+  if (!win_score || !kept || !idx) return PC_ERR_INVALID_ARG;
+  if (C < 1 || m < 1 || m > C || Hkv < 1 || L < 1 || n_cand < 1 || n_cand > L || k < 1) return PC_ERR_INVALID_ARG;
+  if (n_s < 0 || n_r < 0 || lambda_s != lambda_s || lambda_m != lambda_m || lambda_r != lambda_r) return PC_ERR_INVALID_ARG;
+  if (n_cand > 32768) return PC_ERR_UNSUPPORTED;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  const float calib[5] = {(float)n_s, (float)n_r, lambda_s, lambda_m, lambda_r};
+  if (pc::launch_select_tokens(win_score, kept, m, Hkv, L, n_cand, k, idx, calib, static_cast<cudaStream_t>(stream)) !=
+      cudaSuccess)
     return PC_ERR_CUDA;
   return PC_OK;
 }

@@ -16,8 +16,9 @@ void launch_rope_keys(const void* k, const long long k_stride[3], void* k_rot, c
 // ---- pc_select_gather.cu
 void launch_chunk_score(const float* win_lse, int C, int n_per_chunk, float* score, cudaStream_t st);
 void launch_select_chunks(const float* score, int C, int m, int lower_is_better, int* kept, cudaStream_t st);
+// calib: null, or host array {n_s, n_r, lam_s, lam_m, lam_r} (attention calibration, Eq. 8)
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
-                                 int* idx, cudaStream_t st);
+                                 int* idx, const float* calib, cudaStream_t st);
 cudaError_t launch_gather_kv(const void* k_src, const void* v_src, const long long stride_elems[3], const int* kept,
                              const int* idx, int m, int Hkv, int k, int d, void* k_out, void* v_out, int* pos_out,
                              int sm_count, cudaStream_t st);

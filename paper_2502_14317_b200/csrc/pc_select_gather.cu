@@ -82,9 +82,17 @@ constexpr int SEL_MAX_THREADS = 1024;                          // n_cand <= 3276
 
 __device__ __forceinline__ int sel_pad(int p) { return p + (p >> 5); }
 
+// Attention calibration (Eq. 8): a candidate whose score exceeds the threshold of its region (first n_s
+// positions / last n_r positions / the rest) is evicted before the ranking.  +inf switches a region off.
+struct SelCalib {
+  int on, n_s, n_r;
+  float lam_s, lam_m, lam_r;
+};
+
 __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const float* __restrict__ win_score,
                                                                         const int* __restrict__ kept, int Hkv, int L,
-                                                                        int n_cand, int k, int* __restrict__ idx) {
+                                                                        int n_cand, int k, int* __restrict__ idx,
+                                                                        const SelCalib cal) {
   extern __shared__ uint32_t sel_smem[];                       // [n_pad] keys, later reused for the staged output
   __shared__ int s_cnt[32];                                    // per bit: keys of the row >= the candidate threshold
   __shared__ int2 s_scan[32];
@@ -95,13 +103,26 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
   int* out = idx + (size_t)row * k;
 
   if (tid < 32) s_cnt[tid] = 0;                                // visible after the barrier that follows the row load
-  if (k >= n_cand) {                                           // nothing to evict: identity, then -1 padding
+  if (k >= n_cand && !cal.on) {                                // nothing to evict: identity, then -1 padding
     for (int j = tid; j < k; j += blockDim.x) out[j] = j < n_cand ? j : -1;
     return;
   }
+  const int k_out = k;
+  if (k > n_cand) k = n_cand;                                  // calibrated: rank all candidates, pad the rest
   const int c = kept[r];
   const float* src = win_score + ((size_t)c * Hkv + hk) * L;
 
+  // keys: NaN ranks below every number (1); evicted candidates and the padding rank below NaN (0) and are
+  // never emitted
+  auto key_of = [&](float v, int p) -> uint32_t {
+    uint32_t kk = rank_key(v, false);
+    kk = kk == 0u ? 1u : kk;
+    if (cal.on) {
+      const float lam = p < cal.n_s ? cal.lam_s : (p >= n_cand - cal.n_r ? cal.lam_r : cal.lam_m);
+      if (v > lam) kk = 0u;
+    }
+    return kk;
+  };
   // ---- 1. row -> shared memory (coalesced), -> registers (32 consecutive positions per thread)
   if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
     const float4* src4 = reinterpret_cast<const float4*>(src);
@@ -110,11 +131,11 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
       const float4 v = __ldg(src4 + i);
       const int p = 4 * i;                                     // 4 consecutive positions never straddle a pad slot
       uint32_t* d = sel_smem + sel_pad(p);
-      d[0] = rank_key(v.x, false); d[1] = rank_key(v.y, false); d[2] = rank_key(v.z, false); d[3] = rank_key(v.w, false);
+      d[0] = key_of(v.x, p); d[1] = key_of(v.y, p + 1); d[2] = key_of(v.z, p + 2); d[3] = key_of(v.w, p + 3);
     }
-    for (int p = (n4 << 2) + tid; p < n_cand; p += blockDim.x) sel_smem[sel_pad(p)] = rank_key(__ldg(src + p), false);
+    for (int p = (n4 << 2) + tid; p < n_cand; p += blockDim.x) sel_smem[sel_pad(p)] = key_of(__ldg(src + p), p);
   } else {
-    for (int p = tid; p < n_cand; p += blockDim.x) sel_smem[sel_pad(p)] = rank_key(__ldg(src + p), false);
+    for (int p = tid; p < n_cand; p += blockDim.x) sel_smem[sel_pad(p)] = key_of(__ldg(src + p), p);
   }
   __syncthreads();
   uint32_t key[SEL_KPT];
@@ -157,7 +178,8 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
       active &= ~key[31 - bit];
     }
   }
-  // active = keys == T (padding keys are 0 and can only tie with NaN keys, which sit at lower positions)
+  // active = keys == T.  T == 0 only when fewer than k candidates survived calibration: the keys equal to 0
+  // are evicted candidates and padding, none of which is emitted
 
   // ---- 3. ordered emission
   const int gt = n_above, eq = __popc(active);
@@ -175,7 +197,8 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
     if (wv < warp) { gt_before += t.x; eq_before += t.y; }
     gt_total += t.x;
   }
-  const int need_eq = k - gt_total;                            // keys equal to T that are taken (lowest positions first)
+  const int need_eq = T == 0u ? 0 : k - gt_total;              // keys equal to T that are taken (lowest positions first)
+  const int n_emit = gt_total + need_eq;
   int* stage = reinterpret_cast<int*>(sel_smem);               // [k]
 #pragma unroll
   for (int i = 0; i < SEL_KPT; ++i) {
@@ -189,16 +212,19 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
     }
   }
   __syncthreads();
-  for (int j = tid; j < k; j += blockDim.x) out[j] = stage[j];
+  for (int j = tid; j < k_out; j += blockDim.x) out[j] = j < n_emit ? stage[j] : -1;
 }
 
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
-                                 int* idx, cudaStream_t st) {
+                                 int* idx, const float* calib /* null or {n_s, n_r, lam_s, lam_m, lam_r} */,
+                                 cudaStream_t st) {
   int threads = ((n_cand + SEL_KPT - 1) / SEL_KPT + 31) / 32 * 32;
   if (threads < 32) threads = 32;
   if (threads > SEL_MAX_THREADS) return cudaErrorInvalidValue;
   const size_t words = (size_t)n_cand + (n_cand >> 5) + 1;
-  const size_t stage = k < n_cand ? (size_t)k : 0;             // k >= n_cand writes the identity directly
+  SelCalib cal = {0, 0, 0, 0.f, 0.f, 0.f};
+  if (calib) cal = SelCalib{1, (int)calib[0], (int)calib[1], calib[2], calib[3], calib[4]};
+  const size_t stage = (k < n_cand || cal.on) ? (size_t)(k < n_cand ? k : n_cand) : 0;   // uncalibrated k >= n_cand writes the identity directly
   const size_t smem = (words > stage ? words : stage) * sizeof(uint32_t);
   static size_t configured = 0;
   if (smem > 48 * 1024 && smem > configured) {
@@ -206,7 +232,7 @@ cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m,
     if (e != cudaSuccess) return e;
     configured = smem;
   }
-  select_tokens_kernel<<<m * Hkv, threads, smem, st>>>(win_score, kept, Hkv, L, n_cand, k, idx);
+  select_tokens_kernel<<<m * Hkv, threads, smem, st>>>(win_score, kept, Hkv, L, n_cand, k, idx, cal);
   return cudaGetLastError();
 }
 

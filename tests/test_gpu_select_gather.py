@@ -103,3 +103,31 @@ def test_keep_all_gather_is_a_reshape():
     idx = pc.select_tokens(_dev(S), kept, ctx, ctx)
     kc, vc, pos = pc.gather_kv(to_dev(k_rot), to_dev(k_rot), kept, idx)
     assert np.array_equal(to_bits(kc), k_rot[:, :ctx].transpose(2, 0, 1, 3).reshape(Hkv, C * ctx, d))
+
+
+@pytest.mark.parametrize("C,m,L,w,k,Hkv,n_s,n_r,lams", [
+    (3, 2, 600, 8, 100, 2, 100, 100, (0.6, 0.9, 0.4)),          # all three regions active
+    (2, 2, 300, 16, 284, 2, 10, 20, (0.5, 0.5, 0.5)),           # k = n_cand: survivors only, -1 padding
+    (2, 1, 8192, 64, 2048, 8, 100, 100, (float("inf"), 0.97, float("inf"))),   # workload row shape, middle peaks only
+    (1, 1, 200, 8, 50, 1, 150, 150, (0.2, 0.3, 0.4)),           # overlapping regions: the sink region wins
+    (2, 2, 400, 8, 30, 2, 100, 100, (0.0, 0.0, 0.0)),           # everything above the thresholds: all -1
+])
+def test_select_tokens_calibrated(C, m, L, w, k, Hkv, n_s, n_r, lams):
+    import paper_2502_14317_b200 as pc
+    rng = np.random.default_rng(L + k)
+    S = rng.random((C, Hkv, L)).astype(np.float32)
+    S[:, :, 0] = 50.0                                            # a sink peak
+    S[:, :, 5] = np.float32(lams[0]) if np.isfinite(lams[0]) else 0.5   # exactly at the threshold: kept
+    S[0, 0, 7] = np.nan
+    kept = np.sort(rng.choice(C, size=m, replace=False)).astype(np.int32)
+    got = pc.select_tokens_calibrated(torch.from_numpy(S).cuda(), torch.from_numpy(kept).cuda(), L - w, k, n_s=n_s,
+                                      n_r=n_r, lambda_s=lams[0], lambda_m=lams[1], lambda_r=lams[2])
+    torch.cuda.synchronize()
+    ref = orc.select_tokens_calibrated(S, kept, L - w, k, n_s, n_r, *lams)
+    assert np.array_equal(got.cpu().numpy(), ref)
+    # thresholds at +inf: the calibrated entry point is pc_select_tokens
+    inf = float("inf")
+    a = pc.select_tokens_calibrated(torch.from_numpy(S).cuda(), torch.from_numpy(kept).cuda(), L - w, k, n_s=n_s, n_r=n_r,
+                                    lambda_s=inf, lambda_m=inf, lambda_r=inf)
+    b = pc.select_tokens(torch.from_numpy(S).cuda(), torch.from_numpy(kept).cuda(), L - w, k)
+    assert torch.equal(a, b)
