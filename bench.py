@@ -386,7 +386,21 @@ def extra_measurements(pc, torch, dev, peaks) -> dict:
                                  "frac_of_measured_bf16_burst": flops / us / 1e6 / peaks["bf16_tflops"],
                                  "frac_of_measured_hbm": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
                                  "flops": flops, "kv_bytes": kv_bytes, "l2": "4.3 GB of K/V per call, larger than L2"}
-    del qw, kc, vc, kw, vw, buf
+    # ---- decoding step over the same caches: one query token per sequence (w = 1), HBM-bound
+    q1 = torch.randn((B, 1, Hq, d), device=dev, generator=g).bfloat16()
+    k1 = torch.randn((B, 1, Hkv, d), device=dev, generator=g).bfloat16()
+    v1 = torch.randn((B, 1, Hkv, d), device=dev, generator=g).bfloat16()
+    buf1 = {}
+
+    def run_dec():
+        r = pc.parallel_attn(q1, kc, vc, k1, v1, q_pos0=8191, rope_theta=5e5, out=buf1.get("out"), status=buf1.get("status"),
+                             workspace=buf1.get("workspace"))
+        buf1.update(r)
+    us = _time_us(torch, run_dec, reps=10)
+    out["decode_step_cfg4_caches"] = {"us": us, "kv_gbs": kv_bytes / us / 1e3,
+                                      "frac_of_measured_hbm": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
+                                      "kv_bytes": kv_bytes, "note": "pc_parallel_attn with w = 1, B = 64, Nk = 16384"}
+    del qw, kc, vc, kw, vw, buf, q1, k1, v1, buf1
     # ---- token top-k, cfg1 row shape (8128 candidates -> 2048) on 65536 rows (2.1 GB of scores)
     C, Hk, L, n_cand, k = 8192, 8, 8192, 8128, 2048
     score = torch.rand((C, Hk, L), device=dev, generator=g)

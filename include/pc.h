@@ -164,6 +164,9 @@ PC_API int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t*
  * keys.  Keys arrive already rotated.  Split over key ranges with an fp32 merge.
  * q_win [B,w,Hq,d]; k_cache, v_cache [B,Hkv,Nk,d]; k_win, v_win [B,w,Hkv,d];
  * out [B,w,Hq,d] bf16; lse_out [B,Hq,w] fp32 natural log (may be NULL).  All contiguous.
+ * Here w may be any power of two in [1, 128]: w = 1 is a decoding step over the compressed
+ * cache (the paper keeps the cache for generation; the new token's own key/value are k_win,
+ * v_win and the caller appends them to the cache afterwards).
  */
 PC_API size_t pc_parallel_attn_workspace_bytes(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk);
 

@@ -271,7 +271,7 @@ ParallelPlan parallel_plan(int B, int w, int Hq, int Hkv, int d, int Nk, int sm_
 int32_t check_parallel_args(int B, int w, int Hq, int Hkv, int d, int Nk) {
   if (B < 1 || w < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || Nk < 1) return PC_ERR_INVALID_ARG;
   if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
-  if (!pow2_between(w, 8, 128)) return PC_ERR_UNSUPPORTED;
+  if (!pow2_between(w, 1, 128)) return PC_ERR_UNSUPPORTED;      // w = 1: one new token decoding over the cache
   if ((long long)B * Hq > (1 << 24) || Nk > (1 << 28)) return PC_ERR_UNSUPPORTED;
   return PC_OK;
 }

@@ -69,6 +69,7 @@ def test_host_side_argument_errors_need_no_gpu(lib):
     assert lib.pc_select_tokens(p, o, 4, 2, 2, 256, 300, 64, o, None) == -1    # n_cand > L
     assert lib.pc_gather_kv(p, p, None, 256, o, o, 2, 2, 64, 96, p, p, None, None) == -2   # head size
     assert lib.pc_parallel_attn(1, 24, 4, 2, 64, 128, p, 0, 1e4, 0.0, p, p, p, p, p, None, None, None, 0, None) == -2
+    assert lib.pc_select_tokens_calibrated(p, o, 4, 2, 2, 256, 200, 64, -1, 0, 1.0, 1.0, 1.0, o, None) == -1   # n_s < 0
 
 
 def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):

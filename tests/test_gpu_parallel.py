@@ -22,6 +22,9 @@ def _bits(rng, shape):
     (1, 64, 8, 1, 128, 700, 8128, 5e5),       # G*w = 512 rows: two row groups per kv-head
     (2, 128, 2, 1, 64, 77, 0, 1e4),           # cache shorter than one tile, widest window
     (1, 32, 6, 2, 128, 2049, 100, 1e4),       # G = 3, one key past a tile boundary
+    (2, 1, 8, 2, 128, 3000, 8191, 5e5),       # decoding step: one query token over the cache (+ its own key)
+    (3, 2, 4, 4, 64, 500, 4094, 1e4),         # two query tokens, MHA
+    (1, 4, 32, 8, 128, 16384, 8188, 5e5),     # four query tokens over a 16K cache, Llama-3 heads
 ])
 def test_parallel_attn_shapes(B, w, Hq, Hkv, d, Nk, q_pos0, theta):
     import paper_2502_14317_b200 as pc
