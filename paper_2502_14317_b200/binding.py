@@ -312,3 +312,57 @@ def hot_path(q, k, v, *, w, rope_theta, m, k_keep, softmax_scale=0.0, chunk_scor
                         "kc": kc, "vc": vc, "pos": pos, "fg": res["fg"], "status": res["status"],
                         "ws_prefill": res["ws_prefill"], "ws_par": res["ws_par"]})
     return res
+
+
+def hot_path_from_host(hq, hk, hv, *, w, rope_theta, m, k_keep, softmax_scale=0.0, n_groups=4, buffers=None):
+    """The whole path for inputs that live in pinned HOST memory (hq [C,L,Hq,d], hk/hv [C,L,Hkv,d], bf16).
+
+    Chunks are independent until the chunk ranking, so they are uploaded in ``n_groups`` groups on a copy
+    stream while the attention of the previous group runs on the current stream; the ranking, gather and
+    parallel attention follow once all groups are done.  ``buffers`` (dict) keeps the device tensors,
+    streams and events between calls.  Returns the same dict as :func:`hot_path` (device tensors).
+    """
+    b = {} if buffers is None else buffers
+    C, L, Hq, d = hq.shape
+    Hkv = hk.shape[2]
+    dev = torch.device("cuda", torch.cuda.current_device())
+    if "q" not in b:
+        b["q"] = torch.empty(hq.shape, dtype=torch.bfloat16, device=dev)
+        b["k"] = torch.empty(hk.shape, dtype=torch.bfloat16, device=dev)
+        b["v"] = torch.empty(hv.shape, dtype=torch.bfloat16, device=dev)
+        b["o"] = torch.empty(hq.shape, dtype=torch.bfloat16, device=dev)
+        b["k_rot"] = torch.empty(hk.shape, dtype=torch.bfloat16, device=dev)
+        b["win_score"] = torch.empty((C, Hkv, L), dtype=torch.float32, device=dev)
+        b["win_lse"] = torch.empty((C, Hq, w), dtype=torch.float32, device=dev)
+        b["status"] = torch.zeros(1, dtype=torch.int32, device=dev)
+        b["copy_stream"] = torch.cuda.Stream(device=dev)
+        b["uploaded"] = [torch.cuda.Event() for _ in range(n_groups)]
+        b["consumed"] = torch.cuda.Event()
+    q, k, v = b["q"], b["k"], b["v"]
+    main, copy = torch.cuda.current_stream(), b["copy_stream"]
+    copy.wait_stream(main)                       # the previous call may still read q, k, v
+    bounds = [(g * C) // n_groups for g in range(n_groups + 1)]
+    for g in range(n_groups):
+        c0, c1 = bounds[g], bounds[g + 1]
+        if c1 == c0:
+            continue
+        with torch.cuda.stream(copy):
+            q[c0:c1].copy_(hq[c0:c1], non_blocking=True)
+            k[c0:c1].copy_(hk[c0:c1], non_blocking=True)
+            v[c0:c1].copy_(hv[c0:c1], non_blocking=True)
+            b["uploaded"][g].record(copy)
+        main.wait_event(b["uploaded"][g])
+        pre = chunk_prefill_attn(q[c0:c1], k[c0:c1], v[c0:c1], w=w, rope_theta=rope_theta, softmax_scale=softmax_scale,
+                                 out=b["o"][c0:c1], k_rot=b["k_rot"][c0:c1], win_score=b["win_score"][c0:c1],
+                                 win_lse=b["win_lse"][c0:c1], status=b["status"], workspace=b.get("ws_prefill"))
+        b["ws_prefill"] = pre["workspace"]
+    score = chunk_score_from_lse(b["win_lse"], out=b.get("chunk_score"))
+    kept = select_chunks(score, m, True, out=b.get("kept"))
+    idx = select_tokens(b["win_score"], kept, L - w, k_keep, out=b.get("idx"))
+    kc, vc, pos = gather_kv(b["k_rot"], v, kept, idx, k_out=b.get("kc"), v_out=b.get("vc"), pos_out=b.get("pos"))
+    pa = parallel_attn(q[0:1, L - w:], kc.unsqueeze(0), vc.unsqueeze(0), b["k_rot"][0:1, L - w:], v[0:1, L - w:],
+                       q_pos0=L - w, rope_theta=rope_theta, softmax_scale=softmax_scale, out=b.get("fg"),
+                       status=b["status"], workspace=b.get("ws_par"))
+    b.update(chunk_score=score, kept=kept, idx=idx, kc=kc, vc=vc, pos=pos, fg=pa["out"], ws_par=pa["workspace"])
+    return {"o": b["o"], "k_rot": b["k_rot"], "win_score": b["win_score"], "win_lse": b["win_lse"], "chunk_score": score,
+            "kept": kept, "idx": idx, "kc": kc, "vc": vc, "pos": pos, "fg": pa["out"], "status": b["status"]}

@@ -109,3 +109,20 @@ def test_single_chunk_keep_all_equals_local_attention():
     assert np.abs(o_win - fg).max() <= 1e-2          # two bf16 roundings of the same quantity
     O, _, _ = orc.local_attention(q, k, v, 1e4)
     check_attention_output(fg, O[0, L - w:], "Fg vs full causal attention")
+
+
+def test_hot_path_from_host_matches_device_path(cfg0_inputs):
+    """Uploading the chunks in groups on a copy stream must give exactly what the all-on-device path gives."""
+    import paper_2502_14317_b200 as pc
+    cfg, inp = cfg0_inputs
+    pin = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hq, hk, hv = pin(inp["q"]), pin(inp["k"]), pin(inp["v"])
+    ref = pc.hot_path(hq.cuda(), hk.cuda(), hv.cuda(), w=cfg.w, rope_theta=cfg.rope_theta, m=cfg.m, k_keep=cfg.k)
+    buffers = {}
+    for _ in range(2):                                            # second call reuses buffers, streams and events
+        got = pc.hot_path_from_host(hq, hk, hv, w=cfg.w, rope_theta=cfg.rope_theta, m=cfg.m, k_keep=cfg.k, n_groups=3,
+                                    buffers=buffers)
+        torch.cuda.synchronize()
+        assert int(got["status"].item()) == 0
+        for key in ("o", "k_rot", "win_score", "win_lse", "kept", "idx", "kc", "vc", "fg"):
+            assert torch.equal(got[key], ref[key]), key
