@@ -64,23 +64,25 @@ void launch_select_chunks(const float* score, int C, int m, int lower_is_better,
 }
 
 // ------------------------------------------------------------------ token top-k
-// One CTA per (kept chunk, kv-head) row, 32 candidates per thread held in REGISTERS.
-//   1. The row is read once with coalesced 16-byte loads into shared memory (padded by one
-//      word per 32 so that the next step is free of bank conflicts); every thread then takes
-//      the 32 consecutive positions [32 tid, 32 tid + 32) as order-preserving uint32 keys and
-//      transposes its 32 x 32 bit matrix in registers: word b then holds bit b of all 32 keys.
+// One CTA per (kept chunk, kv-head) row, 32 candidates per thread held in REGISTERS, no staging
+// of the row in shared memory.
+//   1. Warp w owns the 1024 positions [1024 w, 1024 w + 1024).  Lane l reads them as 8 coalesced
+//      16-byte loads (chunk j = positions 1024 w + 128 j + 4 l + 0..3), turns every score into an
+//      order-preserving uint32 key and transposes its 32 x 32 bit matrix in registers: word b then
+//      holds bit b of all 32 keys (byte permutes for the 16- and 8-bit stages).
 //   2. The k-th largest key T is found bit by bit, most significant first.  On the bit slices a
-//      round is three instructions per thread (and, popc, add) plus one redux per warp, one
-//      shared-memory atomic per warp and one barrier: 32 rounds whatever the distribution of
-//      the scores, no histogram hot spots, and the masks of the keys > T and == T fall out.
-//   3. One block scan of (count > T, count == T) gives every thread its output offset; positions
-//      with key > T plus the first (k - count_gt) positions with key == T are staged in shared
-//      memory in ascending order (ties go to the lower position) and written out coalesced.
+//      round is three instructions per thread (and, popc, redux) plus one shared-memory atomic
+//      per warp and one barrier, whatever the distribution of the scores; the masks of the keys
+//      > T and == T fall out.  The search stops as soon as every key still undecided belongs to
+//      the top k (with distinct scores after about log2(n_cand) rounds past their common prefix).
+//   3. One block scan over the per-chunk counts (eight counts packed in two words) gives every
+//      thread the output rank of its kept positions, which are stored straight to the index row in
+//      ascending order.  Only when the keys equal to T cannot all be kept does a second scan rank
+//      them first (ties go to the lower position).
 // HBM traffic: the row once (4 B per candidate) + 4 B per kept index.
 constexpr int SEL_KPT = 32;                                    // keys per thread
+constexpr int SEL_SPAN = 32 * SEL_KPT;                         // positions per warp
 constexpr int SEL_MAX_THREADS = 1024;                          // n_cand <= 32768
-
-__device__ __forceinline__ int sel_pad(int p) { return p + (p >> 5); }
 
 // Attention calibration (Eq. 8): a candidate whose score exceeds the threshold of its region (first n_s
 // positions / last n_r positions / the rest) is evicted before the ranking.  +inf switches a region off.
@@ -89,21 +91,60 @@ struct SelCalib {
   float lam_s, lam_m, lam_r;
 };
 
+// 4 nibbles of a 16-bit value -> 4 bytes
+__device__ __forceinline__ uint32_t sel_spread_nibbles(uint32_t h) {
+  const uint32_t t = (h | (h << 8)) & 0x00FF00FFu;
+  return (t | (t << 4)) & 0x0F0F0F0Fu;
+}
+
+// Ranks in position order.  Bit 31 - i of x belongs to key i of the thread (chunk j = i / 4).  On return
+// offs[j] is the number of set bits of the whole block at positions before this thread's chunk j; the
+// return value is the number of set bits of the block.  Contains one block barrier.
+__device__ __forceinline__ int sel_ordered_offsets(uint32_t x, int lane, int warp, int nwarps, int* s_tot,
+                                                   int (&offs)[8]) {
+  uint32_t n = x - ((x >> 1) & 0x55555555u);
+  n = (n & 0x33333333u) + ((n >> 2) & 0x33333333u);            // per nibble: its population count
+  const uint32_t own_hi = sel_spread_nibbles(n >> 16);         // byte 3 - j: chunk j (j < 4)
+  const uint32_t own_lo = sel_spread_nibbles(n & 0xFFFFu);     // byte 7 - j: chunk j (j >= 4)
+  uint32_t hi = own_hi, lo = own_lo;                           // inclusive scan over the lanes; a byte holds at most 128
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t a = __shfl_up_sync(0xFFFFFFFFu, hi, off), b = __shfl_up_sync(0xFFFFFFFFu, lo, off);
+    if (lane >= off) { hi += a; lo += b; }
+  }
+  const uint32_t t_hi = __shfl_sync(0xFFFFFFFFu, hi, 31), t_lo = __shfl_sync(0xFFFFFFFFu, lo, 31);
+  const uint32_t e_hi = hi - own_hi, e_lo = lo - own_lo;
+  int run = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int sh = 8 * (3 - (j & 3));
+    offs[j] = run + (int)(((j < 4 ? e_hi : e_lo) >> sh) & 0xFFu);
+    run += (int)(((j < 4 ? t_hi : t_lo) >> sh) & 0xFFu);
+  }
+  if (lane == 0) s_tot[warp] = run;
+  __syncthreads();
+  const int v = lane < nwarps ? s_tot[lane] : 0;
+  const int base = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? v : 0);
+  const int total = __reduce_add_sync(0xFFFFFFFFu, v);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) offs[j] += base;
+  return total;
+}
+
+template <bool CAL>
 __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const float* __restrict__ win_score,
                                                                         const int* __restrict__ kept, int Hkv, int L,
                                                                         int n_cand, int k, int* __restrict__ idx,
                                                                         const SelCalib cal) {
-  extern __shared__ uint32_t sel_smem[];                       // [n_pad] keys, later reused for the staged output
-  __shared__ int s_cnt[32];                                    // per bit: keys of the row >= the candidate threshold
-  __shared__ int2 s_scan[32];
+  __shared__ int s_cnt[32];                                    // per bit: undecided keys of the row with that bit set
+  __shared__ int s_tot[2][32];
 
   const int row = blockIdx.x;                                  // r * Hkv + hkv
   const int r = row / Hkv, hk = row % Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   int* out = idx + (size_t)row * k;
 
-  if (tid < 32) s_cnt[tid] = 0;                                // visible after the barrier that follows the row load
-  if (k >= n_cand && !cal.on) {                                // nothing to evict: identity, then -1 padding
+  if (!CAL && k >= n_cand) {                                   // nothing to evict: identity, then -1 padding
     for (int j = tid; j < k; j += blockDim.x) out[j] = j < n_cand ? j : -1;
     return;
   }
@@ -112,127 +153,155 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
   const int c = kept[r];
   const float* src = win_score + ((size_t)c * Hkv + hk) * L;
 
-  // keys: NaN ranks below every number (1); evicted candidates and the padding rank below NaN (0) and are
-  // never emitted
-  auto key_of = [&](float v, int p) -> uint32_t {
-    uint32_t kk = rank_key(v, false);
-    kk = kk == 0u ? 1u : kk;
-    if (cal.on) {
-      const float lam = p < cal.n_s ? cal.lam_s : (p >= n_cand - cal.n_r ? cal.lam_r : cal.lam_m);
-      if (v > lam) kk = 0u;
-    }
-    return kk;
-  };
-  // ---- 1. row -> shared memory (coalesced), -> registers (32 consecutive positions per thread)
-  if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
-    const float4* src4 = reinterpret_cast<const float4*>(src);
-    const int n4 = n_cand >> 2;
-    for (int i = tid; i < n4; i += blockDim.x) {
-      const float4 v = __ldg(src4 + i);
-      const int p = 4 * i;                                     // 4 consecutive positions never straddle a pad slot
-      uint32_t* d = sel_smem + sel_pad(p);
-      d[0] = key_of(v.x, p); d[1] = key_of(v.y, p + 1); d[2] = key_of(v.z, p + 2); d[3] = key_of(v.w, p + 3);
-    }
-    for (int p = (n4 << 2) + tid; p < n_cand; p += blockDim.x) sel_smem[sel_pad(p)] = key_of(__ldg(src + p), p);
-  } else {
-    for (int p = tid; p < n_cand; p += blockDim.x) sel_smem[sel_pad(p)] = key_of(__ldg(src + p), p);
-  }
-  __syncthreads();
-  uint32_t key[SEL_KPT];
-  const int p0 = tid * SEL_KPT;
+  // ---- 1. the row -> registers
+  const int pbase = warp * SEL_SPAN + 4 * lane;
+  const bool vec = (reinterpret_cast<uintptr_t>(src) & 15u) == 0;
+  float val[SEL_KPT];
+  uint32_t valid = 0u;                                         // bit 31 - i: key i is a candidate
 #pragma unroll
-  for (int i = 0; i < SEL_KPT; ++i) key[i] = (p0 + i < n_cand) ? sel_smem[p0 + i + tid] : 0u;   // pad(p0 + i) = p0 + i + tid; 0 ranks below every candidate
+  for (int j = 0; j < 8; ++j) {
+    const int p = pbase + 128 * j;
+    if (vec && p + 3 < n_cand) {
+      const float4 t = __ldg(reinterpret_cast<const float4*>(src + p));
+      val[4 * j] = t.x; val[4 * j + 1] = t.y; val[4 * j + 2] = t.z; val[4 * j + 3] = t.w;
+      valid |= 0xF0000000u >> (4 * j);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool in = p + e < n_cand;
+        val[4 * j + e] = in ? __ldg(src + p + e) : 0.0f;
+        if (in) valid |= 0x80000000u >> (4 * j + e);
+      }
+    }
+  }
+  if (tid < 32) s_cnt[tid] = 0;
+  __syncthreads();                                             // the counters are cleared before the first round adds to them
+
+  // order-preserving keys: -0 ranks as +0 (the addition turns it into +0); NaN ranks below every number
+  // (key 1); positions that are not candidates rank below NaN (key 0) and are never emitted
+  uint32_t key[SEL_KPT];
+  float nan_probe = 0.0f;                                      // NaN if any score is (or after inf - inf: checked exactly below)
+#pragma unroll
+  for (int i = 0; i < SEL_KPT; ++i) {
+    const float f = __fadd_rn(val[i], 0.0f);
+    nan_probe = __fadd_rn(nan_probe, f);
+    const uint32_t u = __float_as_uint(f);
+    key[i] = u ^ (static_cast<uint32_t>(static_cast<int32_t>(u) >> 31) | 0x80000000u);
+    if (CAL) {
+      const int p = pbase + 128 * (i >> 2) + (i & 3);
+      const float lam = p < cal.n_s ? cal.lam_s : (p >= n_cand - cal.n_r ? cal.lam_r : cal.lam_m);
+      if (val[i] > lam) valid &= ~(0x80000000u >> i);
+    }
+  }
+  if (nan_probe != nan_probe) {                                // rare
+#pragma unroll
+    for (int i = 0; i < SEL_KPT; ++i)
+      if (key[i] > 0xFF800000u || key[i] < 0x007FFFFFu) key[i] = 1u;   // the images of +NaN and -NaN
+  }
+  if (valid != 0xFFFFFFFFu) {
+#pragma unroll
+    for (int i = 0; i < SEL_KPT; ++i)
+      if (!(valid & (0x80000000u >> i))) key[i] = 0u;
+  }
 
   // in-register transpose of the 32 x 32 bit matrix: afterwards key[31 - b] holds bit b of every
-  // key, the key at position p0 + i sitting at bit 31 - i
+  // key, key i sitting at bit 31 - i
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {                               // exchange 16-bit halves
+    const uint32_t a = key[q], b = key[q + 16];
+    key[q] = __byte_perm(a, b, 0x3276);                        // (a & 0xFFFF0000) | (b >> 16)
+    key[q + 16] = __byte_perm(a, b, 0x1054);                   // (b & 0x0000FFFF) | (a << 16)
+  }
+#pragma unroll
+  for (int q = 0; q < 32; ++q) {                               // exchange bytes
+    if (q & 8) continue;
+    const uint32_t a = key[q], b = key[q + 8];
+    key[q] = __byte_perm(a, b, 0x3715);                        // (a & 0xFF00FF00) | ((b >> 8) & 0x00FF00FF)
+    key[q + 8] = __byte_perm(a, b, 0x2604);                    // (b & 0x00FF00FF) | ((a << 8) & 0xFF00FF00)
+  }
   {
-    uint32_t m = 0x0000FFFFu;
+    uint32_t m = 0x0F0F0F0Fu;
 #pragma unroll
-    for (int j = 16; j != 0; j >>= 1, m ^= (m << j)) {
+    for (int j = 4; j != 0; j >>= 1, m ^= (m << j)) {
 #pragma unroll
-      for (int q = 0; q < 32; q = (q + j + 1) & ~j) {
-        const uint32_t t = (key[q] ^ (key[q + j] >> j)) & m;
-        key[q] ^= t;
-        key[q + j] ^= (t << j);
+      for (int q = 0; q < 32; ++q) {
+        if (q & j) continue;
+        const uint32_t a = key[q], b = key[q + j];
+        key[q] = (a & ~m) | ((b >> j) & m);
+        key[q + j] = (b & m) | ((a << j) & ~m);
       }
     }
   }
 
-  // ---- 2. k-th largest key, bit by bit.  active: keys equal to T on the bits decided so far;
-  // above: keys already known to be larger than T.
-  uint32_t active = 0xFFFFFFFFu, above = 0u, T = 0u;
-  int n_above = 0;
+  // ---- 2. k-th largest key, bit by bit.  active: keys equal to T on the bits decided so far (n_active of
+  // them in the row, of which the `need` largest are kept); above: keys already known to be larger than T.
+  uint32_t active = 0xFFFFFFFFu, above = 0u;
+  int n_active = SEL_KPT * blockDim.x, need = k;
 #pragma unroll
   for (int bit = 31; bit >= 0; --bit) {
+    if (n_active == need) break;                               // every undecided key is kept
     const uint32_t ones = active & key[31 - bit];
-    int cnt = n_above + __popc(ones);                          // keys >= (T | 1 << bit)
-    cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+    const int cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(ones));
     if (lane == 0) atomicAdd(&s_cnt[bit], cnt);
     __syncthreads();
-    if (s_cnt[bit] >= k) {                                     // at least k keys are that large: the k-th largest has this bit
-      T |= 1u << bit;
+    const int tot = s_cnt[bit];                                // undecided keys with this bit set
+    if (tot >= need) {                                         // the k-th largest has this bit
       active = ones;
+      n_active = tot;
     } else {
       above |= ones;
-      n_above += __popc(ones);
       active &= ~key[31 - bit];
+      need -= tot;
+      n_active -= tot;
     }
   }
-  // active = keys == T.  T == 0 only when fewer than k candidates survived calibration: the keys equal to 0
-  // are evicted candidates and padding, none of which is emitted
 
   // ---- 3. ordered emission
-  const int gt = n_above, eq = __popc(active);
-  int sgt = gt, seq = eq;                                      // inclusive warp scan of both counts
+  uint32_t taken;
+  if (n_active == need) {
+    taken = (above | active) & valid;
+  } else {
+    // all 32 bits decided and more keys equal T than are needed: the lowest positions win.  (When T is 0
+    // the keys equal to it are no candidates, and nothing more is taken.)
+    const uint32_t eq = active & valid;
+    int eq_before[8];
+    sel_ordered_offsets(eq, lane, warp, nwarps, s_tot[1], eq_before);
+    uint32_t pick = 0u;
 #pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const int a = __shfl_up_sync(0xFFFFFFFFu, sgt, off), b2 = __shfl_up_sync(0xFFFFFFFFu, seq, off);
-    if (lane >= off) { sgt += a; seq += b2; }
+    for (int i = 0; i < SEL_KPT; ++i) {
+      const uint32_t sel_bit = 0x80000000u >> i;
+      if (eq & sel_bit) {
+        if (eq_before[i >> 2] < need) pick |= sel_bit;
+        ++eq_before[i >> 2];
+      }
+    }
+    taken = (above & valid) | pick;
   }
-  if (lane == 31) s_scan[warp] = make_int2(sgt, seq);
-  __syncthreads();                                             // also: every thread is done reading the keys from shared memory
-  int gt_before = sgt - gt, eq_before = seq - eq, gt_total = 0;
-  for (int wv = 0; wv < nwarps; ++wv) {
-    const int2 t = s_scan[wv];
-    if (wv < warp) { gt_before += t.x; eq_before += t.y; }
-    gt_total += t.x;
-  }
-  const int need_eq = T == 0u ? 0 : k - gt_total;              // keys equal to T that are taken (lowest positions first)
-  const int n_emit = gt_total + need_eq;
-  int* stage = reinterpret_cast<int*>(sel_smem);               // [k]
+  int offs[8];
+  const int n_emit = sel_ordered_offsets(taken, lane, warp, nwarps, s_tot[0], offs);
 #pragma unroll
   for (int i = 0; i < SEL_KPT; ++i) {
-    const uint32_t sel_bit = 0x80000000u >> i;
-    if (above & sel_bit) {
-      stage[gt_before + min(eq_before, need_eq)] = p0 + i;
-      ++gt_before;
-    } else if (active & sel_bit) {
-      if (eq_before < need_eq) stage[gt_before + eq_before] = p0 + i;
-      ++eq_before;
+    if (taken & (0x80000000u >> i)) {
+      out[offs[i >> 2]] = pbase + 128 * (i >> 2) + (i & 3);
+      ++offs[i >> 2];
     }
   }
-  __syncthreads();
-  for (int j = tid; j < k_out; j += blockDim.x) out[j] = j < n_emit ? stage[j] : -1;
+  for (int j = n_emit + tid; j < k_out; j += blockDim.x) out[j] = -1;
 }
 
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
                                  int* idx, const float* calib /* null or {n_s, n_r, lam_s, lam_m, lam_r} */,
                                  cudaStream_t st) {
-  int threads = ((n_cand + SEL_KPT - 1) / SEL_KPT + 31) / 32 * 32;
+  int threads = (n_cand + SEL_SPAN - 1) / SEL_SPAN * 32;
   if (threads < 32) threads = 32;
   if (threads > SEL_MAX_THREADS) return cudaErrorInvalidValue;
-  const size_t words = (size_t)n_cand + (n_cand >> 5) + 1;
-  SelCalib cal = {0, 0, 0, 0.f, 0.f, 0.f};
-  if (calib) cal = SelCalib{1, (int)calib[0], (int)calib[1], calib[2], calib[3], calib[4]};
-  const size_t stage = (k < n_cand || cal.on) ? (size_t)(k < n_cand ? k : n_cand) : 0;   // uncalibrated k >= n_cand writes the identity directly
-  const size_t smem = (words > stage ? words : stage) * sizeof(uint32_t);
-  static size_t configured = 0;
-  if (smem > 48 * 1024 && smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(select_tokens_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = smem;
+  if (calib) {
+    const SelCalib cal{1, (int)calib[0], (int)calib[1], calib[2], calib[3], calib[4]};
+    select_tokens_kernel<true><<<m * Hkv, threads, 0, st>>>(win_score, kept, Hkv, L, n_cand, k, idx, cal);
+  } else {
+    const SelCalib cal{0, 0, 0, 0.f, 0.f, 0.f};
+    select_tokens_kernel<false><<<m * Hkv, threads, 0, st>>>(win_score, kept, Hkv, L, n_cand, k, idx, cal);
   }
-  select_tokens_kernel<<<m * Hkv, threads, smem, st>>>(win_score, kept, Hkv, L, n_cand, k, idx, cal);
   return cudaGetLastError();
 }
 
