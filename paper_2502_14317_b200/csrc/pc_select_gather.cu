@@ -177,16 +177,18 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
   if (tid < 32) s_cnt[tid] = 0;
   __syncthreads();                                             // the counters are cleared before the first round adds to them
 
-  // order-preserving keys: -0 ranks as +0 (the addition turns it into +0); NaN ranks below every number
-  // (key 1); positions that are not candidates rank below NaN (key 0) and are never emitted
+  // Keys.  The order-preserving image of a score with bit pattern u is u ^ 0x80000000 for u >= 0 and ~u for
+  // u < 0; the exclusive-or is applied to the bit slices inside the search (one operand more of a logic
+  // instruction there), so the registers keep u itself.  -0 ranks as +0 (the addition turns it into +0);
+  // NaN ranks below every number (image 1 = pattern 0xFFFFFFFE); positions that are not candidates rank
+  // below NaN (image 0 = pattern 0xFFFFFFFF) and are never emitted.
   uint32_t key[SEL_KPT];
   float nan_probe = 0.0f;                                      // NaN if any score is (or after inf - inf: checked exactly below)
 #pragma unroll
   for (int i = 0; i < SEL_KPT; ++i) {
     const float f = __fadd_rn(val[i], 0.0f);
     nan_probe = __fadd_rn(nan_probe, f);
-    const uint32_t u = __float_as_uint(f);
-    key[i] = u ^ (static_cast<uint32_t>(static_cast<int32_t>(u) >> 31) | 0x80000000u);
+    key[i] = __float_as_uint(f);
     if (CAL) {
       const int p = pbase + 128 * (i >> 2) + (i & 3);
       const float lam = p < cal.n_s ? cal.lam_s : (p >= n_cand - cal.n_r ? cal.lam_r : cal.lam_m);
@@ -196,16 +198,16 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
   if (nan_probe != nan_probe) {                                // rare
 #pragma unroll
     for (int i = 0; i < SEL_KPT; ++i)
-      if (key[i] > 0xFF800000u || key[i] < 0x007FFFFFu) key[i] = 1u;   // the images of +NaN and -NaN
+      if ((key[i] & 0x7FFFFFFFu) > 0x7F800000u) key[i] = 0xFFFFFFFEu;
   }
   if (valid != 0xFFFFFFFFu) {
 #pragma unroll
     for (int i = 0; i < SEL_KPT; ++i)
-      if (!(valid & (0x80000000u >> i))) key[i] = 0u;
+      if (!(valid & (0x80000000u >> i))) key[i] = 0xFFFFFFFFu;
   }
 
   // in-register transpose of the 32 x 32 bit matrix: afterwards key[31 - b] holds bit b of every
-  // key, key i sitting at bit 31 - i
+  // pattern, key i sitting at bit 31 - i
 #pragma unroll
   for (int q = 0; q < 16; ++q) {                               // exchange 16-bit halves
     const uint32_t a = key[q], b = key[q + 16];
@@ -237,10 +239,12 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
   // them in the row, of which the `need` largest are kept); above: keys already known to be larger than T.
   uint32_t active = 0xFFFFFFFFu, above = 0u;
   int n_active = SEL_KPT * blockDim.x, need = k;
+  const uint32_t neg = key[0];                                 // sign bits: the slices below bit 31 are inverted for these keys
 #pragma unroll
   for (int bit = 31; bit >= 0; --bit) {
     if (n_active == need) break;                               // every undecided key is kept
-    const uint32_t ones = active & key[31 - bit];
+    const uint32_t slice = bit == 31 ? ~neg : key[31 - bit] ^ neg;   // this bit of the order-preserving images
+    const uint32_t ones = active & slice;
     const int cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(ones));
     if (lane == 0) atomicAdd(&s_cnt[bit], cnt);
     __syncthreads();
@@ -250,7 +254,7 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
       n_active = tot;
     } else {
       above |= ones;
-      active &= ~key[31 - bit];
+      active &= ~slice;
       need -= tot;
       n_active -= tot;
     }
@@ -281,10 +285,9 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
   const int n_emit = sel_ordered_offsets(taken, lane, warp, nwarps, s_tot[0], offs);
 #pragma unroll
   for (int i = 0; i < SEL_KPT; ++i) {
-    if (taken & (0x80000000u >> i)) {
-      out[offs[i >> 2]] = pbase + 128 * (i >> 2) + (i & 3);
-      ++offs[i >> 2];
-    }
+    const bool t = (taken & (0x80000000u >> i)) != 0u;
+    if (t) out[offs[i >> 2]] = pbase + 128 * (i >> 2) + (i & 3);
+    offs[i >> 2] += t ? 1 : 0;
   }
   for (int j = n_emit + tid; j < k_out; j += blockDim.x) out[j] = -1;
 }
