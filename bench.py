@@ -361,13 +361,23 @@ def _time_us(torch, fn, warm=3, reps=20):
     return 1e3 * e0.elapsed_time(e1) / reps
 
 
-def extra_measurements(pc, torch, dev, peaks) -> dict:
+def extra_measurements(pc, torch, dev, peaks, only=None, select_chunks=8192) -> dict:
     """Single-call timings of the stages whose full-size workloads are not part of the cfg1 step
     (outside the timed region; random device data, parity is covered by the tests):
     parallel attention over a batch of compressed caches (cfg4), token top-k on enough rows to be
     bandwidth-bound, and the gather at the cfg2 size."""
     out = {}
     g = torch.Generator(device=dev).manual_seed(4)
+    if only in (None, "parallel"):
+        _extra_parallel(pc, torch, dev, peaks, g, out)
+    if only in (None, "select"):
+        _extra_select(pc, torch, dev, peaks, g, out, select_chunks)
+    if only in (None, "gather"):
+        _extra_gather(pc, torch, dev, peaks, g, out)
+    return out
+
+
+def _extra_parallel(pc, torch, dev, peaks, g, out):
     # ---- cfg4: B=64 sequences x (8 kept chunks x 2048 keys), 64 window queries
     B, w, Hq, Hkv, d, Nk = 64, 64, 32, 8, 128, 16384
     qw = torch.randn((B, w, Hq, d), device=dev, generator=g).bfloat16()
@@ -402,18 +412,23 @@ def extra_measurements(pc, torch, dev, peaks) -> dict:
     out["decode_step_cfg4_caches"] = {"us": us, "kv_gbs": kv_bytes / us / 1e3,
                                       "frac_of_measured_hbm": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
                                       "kv_bytes": kv_bytes, "note": "pc_parallel_attn with w = 1, B = 64, Nk = 16384"}
-    del qw, kc, vc, kw, vw, buf, q1, k1, v1, buf1
-    # ---- token top-k, cfg1 row shape (8128 candidates -> 2048) on 65536 rows (2.1 GB of scores)
-    C, Hk, L, n_cand, k = 8192, 8, 8192, 8128, 2048
+
+
+def _extra_select(pc, torch, dev, peaks, g, out, n_chunks):
+    # ---- token top-k, cfg1 row shape (8128 candidates -> 2048) on 8 rows per chunk (65536 rows = 2.1 GB of scores)
+    C, Hk, L, n_cand, k = n_chunks, 8, 8192, 8128, 2048
     score = torch.rand((C, Hk, L), device=dev, generator=g)
     kept = torch.arange(C, device=dev, dtype=torch.int32)
     idx = torch.empty((C, Hk, k), device=dev, dtype=torch.int32)
     us = _time_us(torch, lambda: pc.select_tokens(score, kept, n_cand, k, out=idx), reps=5)
     sel_bytes = 4.0 * C * Hk * (n_cand + k)
-    out["select_tokens_65536_rows"] = {"us": us, "algorithmic_bytes": sel_bytes, "gbs": sel_bytes / us / 1e3,
+    out["select_tokens_%d_rows" % (C * Hk)] = {"us": us, "algorithmic_bytes": sel_bytes, "gbs": sel_bytes / us / 1e3,
                                        "frac_of_measured_hbm": sel_bytes / us / 1e3 / peaks["hbm_gbs"]}
-    del score, idx
+
+
+def _extra_gather(pc, torch, dev, peaks, g, out):
     # ---- gather at the cfg2 size: 12 kept chunks x 1024 tokens x 32 heads (201 MB read + 201 MB written)
+    d = 128
     C2, L2, H2, m2, k2 = 32, 4096, 32, 12, 1024
     ksrc = torch.randn((C2, L2, H2, d), device=dev, generator=g).bfloat16()
     vsrc = torch.randn((C2, L2, H2, d), device=dev, generator=g).bfloat16()
@@ -428,7 +443,6 @@ def extra_measurements(pc, torch, dev, peaks) -> dict:
     out["gather_cfg2"] = {"us": us, "algorithmic_bytes": g_bytes, "gbs": g_bytes / us / 1e3,
                           "frac_of_measured_hbm": g_bytes / us / 1e3 / peaks["hbm_gbs"],
                           "l2": "sources 2 x 1.07 GB, larger than L2"}
-    return out
 
 
 def main():
@@ -440,6 +454,10 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the single-call timings of cfg4 / scaled select / cfg2 gather")
+    ap.add_argument("--extra-only", default=None, choices=["parallel", "select", "gather"],
+                    help="run only that single-call measurement and print it (no step loop; e.g. for an ncu capture)")
+    ap.add_argument("--select-chunks", type=int, default=8192,
+                    help="rows / 8 of the scaled token top-k measurement (smaller for an ncu capture)")
     ap.add_argument("--chunks", type=int, default=None,
                     help="override the number of chunks (smaller case of the same workload, e.g. for an ncu capture)")
     ap.add_argument("--traffic-bytes", type=float, default=None,
@@ -450,6 +468,14 @@ def main():
     if args.chunks is not None:
         cfg = dataclasses.replace(cfg, name=f"{cfg.name}[C={args.chunks}]", C=args.chunks, m=min(cfg.m, args.chunks),
                                   n_planted_chunks=min(cfg.n_planted_chunks, args.chunks))
+    if args.extra_only:
+        import torch
+        import paper_2502_14317_b200 as pc
+        dev = torch.device("cuda:0")
+        torch.cuda.set_device(dev)
+        print(json.dumps({"extra": extra_measurements(pc, torch, dev, load_peaks(), only=args.extra_only,
+                                                      select_chunks=args.select_chunks)}))
+        return
     if args.impl == "reference":
         # the oracle takes ~20 s per sample: bound the run to a few minutes whatever K and W say
         args.steps_ref = max(1, min(args.steps, 3))

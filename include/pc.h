@@ -156,6 +156,51 @@ PC_API int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t*
                      void* k_out, void* v_out, int32_t* pos_out, void* stream);
 
 /* ------------------------------------------------------------------------------------
+ * Online chunk queue.  Paper: Sec. 3.1 "Chunk eviction" (the kept chunks live in a priority
+ * queue of fixed size so that prefilling stays inside the memory limit) together with
+ * "Parallel KV cache eviction" applied to every chunk as it is produced (Sec. 5.5
+ * "Throughput analysis": more chunks fit because only compressed caches persist).
+ *
+ * The chunks of a long input arrive in batches.  For every batch the caller runs
+ * pc_chunk_prefill_attn, scores the chunks, runs pc_select_tokens over ALL chunks of the
+ * batch (kept = 0..Cb-1), then
+ *   pc_queue_update  decides which of the m queued chunks and Cb new chunks stay: the m best
+ *                    scores (lowest if lower_is_better != 0; ties go to the lower chunk id;
+ *                    NaN ranks worst; empty slots rank below everything).  A chunk that stays
+ *                    keeps its slot.  slot_src[s] = index within the batch of the chunk that
+ *                    takes over slot s, or -1 where slot s keeps its contents.
+ *   pc_queue_gather  copies the compressed cache of the chunks that moved in:
+ *                        q_k[hkv, s*k + t, :] = k_src[c, idx[c,hkv,t], hkv, :],  c = slot_src[s] >= 0
+ *                    (same for q_v; q_pos[hkv, s*k + t] = idx[c,hkv,t]); other slots are not touched.
+ *                    After it the batch's full K/V may be overwritten by the next batch.
+ * After the last batch pc_queue_emit lists the surviving chunk ids in ascending order in
+ * kept_out[m] (slot_order[m] = their slots) and writes the compressed cache in that order,
+ *     k_out[hkv, i*k + t, :] = q_k[hkv, slot_order[i]*k + t, :]   (same for v_out, pos_out),
+ * which is bit for bit what pc_select_chunks + pc_select_tokens + pc_gather_kv give on all
+ * chunks at once.  If fewer than m chunks were ever pushed the tail of kept_out and
+ * slot_order is -1 and the corresponding rows are zero with position -1.
+ *
+ * State, owned by the caller and living on the device: q_score[m] fp32, q_chunk[m] int32
+ * (chunk id, -1 = empty; set by pc_queue_init), q_k and q_v [Hkv, m*k, d] bf16,
+ * q_pos [Hkv, m*k] int32.  chunk_score[Cb] is a device array; chunk ids of a batch are
+ * chunk_id0 .. chunk_id0 + Cb - 1 and must be unique over the stream.  k_src, v_src, idx,
+ * kv_stride as in pc_gather_kv with idx of shape [Cb,Hkv,k].  Limits: m + Cb <= 1024,
+ * d in {64, 128}, 16-byte aligned K/V pointers.  Everything is enqueued on `stream`.
+ */
+PC_API int32_t pc_queue_init(int32_t m, float* q_score, int32_t* q_chunk, void* stream);
+
+PC_API int32_t pc_queue_update(const float* chunk_score, int32_t Cb, int32_t chunk_id0, int32_t lower_is_better,
+                        int32_t m, float* q_score, int32_t* q_chunk, int32_t* slot_src, void* stream);
+
+PC_API int32_t pc_queue_gather(const void* k_src, const void* v_src, const int64_t* kv_stride, int32_t L,
+                        const int32_t* slot_src, const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d,
+                        void* q_k, void* q_v, int32_t* q_pos, void* stream);
+
+PC_API int32_t pc_queue_emit(const int32_t* q_chunk, int32_t m, int32_t Hkv, int32_t k, int32_t d, const void* q_k,
+                      const void* q_v, const int32_t* q_pos, int32_t* kept_out, int32_t* slot_order, void* k_out,
+                      void* v_out, int32_t* pos_out, void* stream);
+
+/* ------------------------------------------------------------------------------------
  * Parallel (global) attention of the query window over the compressed multi-chunk
  * cache.  Paper: Sec. 3.1 "Global attention", Eq. 9-11.
  * For each of B sequences: the w window queries (rotated here at positions

@@ -59,6 +59,15 @@ def load_library():
     lib.pc_gather_kv.restype = c_int32
     lib.pc_gather_kv.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_int32, c_void_p, c_void_p] + [c_int32] * 4 + \
                                 [c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.pc_queue_init.restype = c_int32
+    lib.pc_queue_init.argtypes = [c_int32, c_void_p, c_void_p, c_void_p]
+    lib.pc_queue_update.restype = c_int32
+    lib.pc_queue_update.argtypes = [c_void_p] + [c_int32] * 4 + [c_void_p] * 4
+    lib.pc_queue_gather.restype = c_int32
+    lib.pc_queue_gather.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_int32, c_void_p, c_void_p] + [c_int32] * 4 + \
+        [c_void_p] * 4
+    lib.pc_queue_emit.restype = c_int32
+    lib.pc_queue_emit.argtypes = [c_void_p] + [c_int32] * 4 + [c_void_p] * 9
     lib.pc_parallel_attn_workspace_bytes.restype = c_size_t
     lib.pc_parallel_attn_workspace_bytes.argtypes = [c_int32] * 6
     lib.pc_parallel_attn.restype = c_int32
@@ -219,6 +228,69 @@ def gather_kv(k_src, v_src, kept, idx, k_out=None, v_out=None, pos_out=None, wan
     return k_out, v_out, pos_out
 
 
+def queue_init(m, Hkv, k, d, device):
+    """pc_queue_init: an empty online chunk queue of m slots with its slot storage.
+
+    Returns the state dict {q_score [m] f32, q_chunk [m] i32, q_k, q_v [Hkv, m*k, d] bf16, q_pos [Hkv, m*k] i32,
+    slot_src [m] i32}."""
+    lib = load_library()
+    st = {"q_score": torch.empty(m, dtype=torch.float32, device=device),
+          "q_chunk": torch.empty(m, dtype=torch.int32, device=device),
+          "q_k": torch.empty((Hkv, m * k, d), dtype=torch.bfloat16, device=device),
+          "q_v": torch.empty((Hkv, m * k, d), dtype=torch.bfloat16, device=device),
+          "q_pos": torch.empty((Hkv, m * k), dtype=torch.int32, device=device),
+          "slot_src": torch.empty(m, dtype=torch.int32, device=device),
+          "m": m, "Hkv": Hkv, "k": k, "d": d}
+    _need_cuda(st["q_score"])
+    _check(lib.pc_queue_init(m, _ptr(st["q_score"]), _ptr(st["q_chunk"]), _stream()), "pc_queue_init")
+    return st
+
+
+def queue_update(state, chunk_score, chunk_id0, lower_is_better=True):
+    """pc_queue_update: push the scores of a batch of chunks (ids chunk_id0, chunk_id0 + 1, ...); fills state['slot_src']."""
+    lib = load_library()
+    _need_cuda(chunk_score)
+    if chunk_score.dtype != torch.float32 or not chunk_score.is_contiguous():
+        raise PcError("chunk_score must be contiguous float32")
+    _check(lib.pc_queue_update(_ptr(chunk_score), chunk_score.numel(), int(chunk_id0), 1 if lower_is_better else 0,
+                               state["m"], _ptr(state["q_score"]), _ptr(state["q_chunk"]), _ptr(state["slot_src"]),
+                               _stream()), "pc_queue_update")
+    return state["slot_src"]
+
+
+def queue_gather(state, k_src, v_src, idx):
+    """pc_queue_gather: move the compressed caches of the chunks that entered the queue into their slots.
+
+    k_src/v_src [Cb,L,Hkv,d] bf16 (rotated keys, values of the batch), idx [Cb,Hkv,k] from select_tokens on all chunks."""
+    lib = load_library()
+    _need_cuda(k_src, v_src, idx)
+    Cb, L, Hkv, d = k_src.shape
+    if idx.shape != (Cb, Hkv, state["k"]) or Hkv != state["Hkv"] or d != state["d"]:
+        raise PcError("idx must be [Cb, Hkv, k] for the queue's k; Hkv and d must match the queue")
+    if k_src.stride() != v_src.stride() or k_src.stride(3) != 1:
+        raise PcError("k_src and v_src must share strides with a contiguous head dimension")
+    strides = (c_int64 * 3)(k_src.stride(0), k_src.stride(1), k_src.stride(2))
+    _check(lib.pc_queue_gather(_ptr(k_src), _ptr(v_src), strides, L, _ptr(state["slot_src"]), _ptr(idx), state["m"], Hkv,
+                               state["k"], d, _ptr(state["q_k"]), _ptr(state["q_v"]), _ptr(state["q_pos"]), _stream()),
+           "pc_queue_gather")
+
+
+def queue_emit(state, k_out=None, v_out=None, pos_out=None, kept_out=None):
+    """pc_queue_emit: the surviving chunks in ascending id order -> (kept [m], k_out, v_out [Hkv, m*k, d], pos [Hkv, m*k])."""
+    lib = load_library()
+    m, Hkv, k, d = state["m"], state["Hkv"], state["k"], state["d"]
+    dev = state["q_k"].device
+    k_out = torch.empty((Hkv, m * k, d), dtype=torch.bfloat16, device=dev) if k_out is None else k_out
+    v_out = torch.empty((Hkv, m * k, d), dtype=torch.bfloat16, device=dev) if v_out is None else v_out
+    pos_out = torch.empty((Hkv, m * k), dtype=torch.int32, device=dev) if pos_out is None else pos_out
+    kept_out = torch.empty(m, dtype=torch.int32, device=dev) if kept_out is None else kept_out
+    order = state.setdefault("slot_order", torch.empty(m, dtype=torch.int32, device=dev))
+    _check(lib.pc_queue_emit(_ptr(state["q_chunk"]), m, Hkv, k, d, _ptr(state["q_k"]), _ptr(state["q_v"]),
+                             _ptr(state["q_pos"]), _ptr(kept_out), _ptr(order), _ptr(k_out), _ptr(v_out), _ptr(pos_out),
+                             _stream()), "pc_queue_emit")
+    return kept_out, k_out, v_out, pos_out
+
+
 def parallel_attn_workspace_bytes(B, w, Hq, Hkv, d, Nk) -> int:
     return int(load_library().pc_parallel_attn_workspace_bytes(B, w, Hq, Hkv, d, Nk))
 
@@ -312,6 +384,60 @@ def hot_path(q, k, v, *, w, rope_theta, m, k_keep, softmax_scale=0.0, chunk_scor
                         "kc": kc, "vc": vc, "pos": pos, "fg": res["fg"], "status": res["status"],
                         "ws_prefill": res["ws_prefill"], "ws_par": res["ws_par"]})
     return res
+
+
+def hot_path_streaming(q, k, v, *, w, rope_theta, m, k_keep, batch, softmax_scale=0.0, chunk_score=None, buffers=None):
+    """The whole path with the chunks taken ``batch`` at a time through the online chunk queue.
+
+    Per batch: chunk-local attention, token eviction on EVERY chunk of the batch, queue update, and the
+    compressed caches of the chunks that entered the queue are copied into their slots; the batch's outputs
+    (attention output, rotated keys, window scores) live in buffers of batch size that the next batch
+    overwrites, so device memory beyond the inputs is O(batch + m) chunks whatever C is.  After the last batch
+    the queue is emitted in chunk order and the window attends over it.  Same results as :func:`hot_path`
+    (kept chunks, indices and compressed cache bit for bit).  q, k, v here are whole device tensors
+    [C,L,*,d]; a caller that streams from elsewhere makes the same calls on its own batches.
+    """
+    b = {} if buffers is None else buffers
+    C, L, Hq, d = q.shape
+    Hkv = k.shape[2]
+    dev = q.device
+    if "queue" not in b:
+        b["queue"] = queue_init(m, Hkv, k_keep, d, dev)
+        b["ids"] = torch.arange(batch, dtype=torch.int32, device=dev)
+    else:
+        lib = load_library()
+        _check(lib.pc_queue_init(m, _ptr(b["queue"]["q_score"]), _ptr(b["queue"]["q_chunk"]), _stream()), "pc_queue_init")
+    qu = b["queue"]
+    pre = None
+    for c0 in range(0, C, batch):
+        c1 = min(c0 + batch, C)
+        n = c1 - c0
+        tag = "full" if n == batch else "tail"                 # a shorter last batch has buffers of its own
+        pb = b.setdefault("pre_" + tag, {})
+        pre = chunk_prefill_attn(q[c0:c1], k[c0:c1], v[c0:c1], w=w, rope_theta=rope_theta, softmax_scale=softmax_scale,
+                                 out=pb.get("o"), k_rot=pb.get("k_rot"), win_score=pb.get("win_score"),
+                                 win_lse=pb.get("win_lse"), status=b.get("status"), workspace=pb.get("workspace"))
+        b["status"] = pre["status"]
+        pb.update({"o": pre["o"], "k_rot": pre["k_rot"], "win_score": pre["win_score"], "win_lse": pre["win_lse"],
+                   "workspace": pre["workspace"]})
+        score = chunk_score[c0:c1] if chunk_score is not None else chunk_score_from_lse(pre["win_lse"], out=pb.get("score"))
+        pb["score"] = score if chunk_score is None else pb.get("score")
+        idx = select_tokens(pre["win_score"], b["ids"][:n], L - w, k_keep, out=pb.get("idx"))
+        pb["idx"] = idx
+        queue_update(qu, score, c0, True)
+        queue_gather(qu, pre["k_rot"], v[c0:c1], idx)
+    kept, kc, vc, pos = queue_emit(qu, k_out=b.get("kc"), v_out=b.get("vc"), pos_out=b.get("pos"), kept_out=b.get("kept"))
+    b.update({"kc": kc, "vc": vc, "pos": pos, "kept": kept})
+    q_win = q[0:1, L - w:]
+    q_win = q_win if q_win.is_contiguous() else q_win.contiguous()
+    k_win = pre["k_rot"][0:1, L - w:]                           # the window is the same in every chunk
+    k_win = k_win if k_win.is_contiguous() else k_win.contiguous()
+    v_win = v[0:1, L - w:]
+    v_win = v_win if v_win.is_contiguous() else v_win.contiguous()
+    pa = parallel_attn(q_win, kc.unsqueeze(0), vc.unsqueeze(0), k_win, v_win, q_pos0=L - w, rope_theta=rope_theta,
+                       softmax_scale=softmax_scale, out=b.get("fg"), status=b["status"], workspace=b.get("ws_par"))
+    b.update({"fg": pa["out"], "ws_par": pa["workspace"]})
+    return {"kept": kept, "kc": kc, "vc": vc, "pos": pos, "fg": pa["out"], "status": b["status"]}
 
 
 def hot_path_from_host(hq, hk, hv, *, w, rope_theta, m, k_keep, softmax_scale=0.0, n_groups=4, buffers=None):

@@ -224,8 +224,63 @@ int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t* kv_str
   if (s[0] <= 0 || s[1] <= 0 || s[2] < d || s[0] % 8 || s[1] % 8 || s[2] % 8) return PC_ERR_INVALID_ARG;
   const DeviceInfo& dev = device_info();
   if (dev.ok != 1) return PC_ERR_UNSUPPORTED;
-  if (pc::launch_gather_kv(k_src, v_src, s, kept, idx, m, Hkv, k, d, k_out, v_out, pos_out, dev.sm_count,
+  if (pc::launch_gather_kv(k_src, v_src, s, kept, idx, m, Hkv, k, d, k_out, v_out, pos_out, dev.sm_count, false,
                            static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return PC_ERR_CUDA;
+  return PC_OK;
+}
+
+// ------------------------------------------------------------------------------------ online chunk queue
+int32_t pc_queue_init(int32_t m, float* q_score, int32_t* q_chunk, void* stream) {
+  if (!q_score || !q_chunk || m < 1) return PC_ERR_INVALID_ARG;
+  if (m > 1023) return PC_ERR_UNSUPPORTED;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  pc::launch_queue_init(q_score, q_chunk, m, static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
+}
+
+int32_t pc_queue_update(const float* chunk_score, int32_t Cb, int32_t chunk_id0, int32_t lower_is_better, int32_t m,
+                        float* q_score, int32_t* q_chunk, int32_t* slot_src, void* stream) {
+  if (!chunk_score || !q_score || !q_chunk || !slot_src || Cb < 1 || m < 1 || chunk_id0 < 0) return PC_ERR_INVALID_ARG;
+  if (chunk_id0 > 0x7FFFFFFF - 1024) return PC_ERR_INVALID_ARG;
+  if ((long long)m + Cb > 1024) return PC_ERR_UNSUPPORTED;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  pc::launch_queue_update(chunk_score, Cb, chunk_id0, lower_is_better, m, q_score, q_chunk, slot_src,
+                          static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
+}
+
+int32_t pc_queue_gather(const void* k_src, const void* v_src, const int64_t* kv_stride, int32_t L,
+                        const int32_t* slot_src, const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d,
+                        void* q_k, void* q_v, int32_t* q_pos, void* stream) {
+  if (!k_src || !v_src || !slot_src || !idx || !q_k || !q_v || !q_pos) return PC_ERR_INVALID_ARG;
+  if (m < 1 || Hkv < 1 || k < 1 || L < 1) return PC_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
+  if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(q_k) || !aligned16(q_v)) return PC_ERR_INVALID_ARG;
+  long long s[3];
+  if (kv_stride) { s[0] = kv_stride[0]; s[1] = kv_stride[1]; s[2] = kv_stride[2]; }
+  else { s[0] = (long long)L * Hkv * d; s[1] = (long long)Hkv * d; s[2] = d; }
+  if (s[0] <= 0 || s[1] <= 0 || s[2] < d || s[0] % 8 || s[1] % 8 || s[2] % 8) return PC_ERR_INVALID_ARG;
+  const DeviceInfo& dev = device_info();
+  if (dev.ok != 1) return PC_ERR_UNSUPPORTED;
+  if (pc::launch_gather_kv(k_src, v_src, s, slot_src, idx, m, Hkv, k, d, q_k, q_v, q_pos, dev.sm_count, true,
+                           static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return PC_ERR_CUDA;
+  return PC_OK;
+}
+
+int32_t pc_queue_emit(const int32_t* q_chunk, int32_t m, int32_t Hkv, int32_t k, int32_t d, const void* q_k,
+                      const void* q_v, const int32_t* q_pos, int32_t* kept_out, int32_t* slot_order, void* k_out,
+                      void* v_out, int32_t* pos_out, void* stream) {
+  if (!q_chunk || !q_k || !q_v || !q_pos || !kept_out || !slot_order || !k_out || !v_out) return PC_ERR_INVALID_ARG;
+  if (m < 1 || Hkv < 1 || k < 1) return PC_ERR_INVALID_ARG;
+  if (m > 1023) return PC_ERR_UNSUPPORTED;
+  if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
+  if (!aligned16(q_k) || !aligned16(q_v) || !aligned16(k_out) || !aligned16(v_out)) return PC_ERR_INVALID_ARG;
+  const DeviceInfo& dev = device_info();
+  if (dev.ok != 1) return PC_ERR_UNSUPPORTED;
+  if (pc::launch_queue_emit(q_chunk, m, Hkv, k, d, q_k, q_v, q_pos, kept_out, slot_order, k_out, v_out, pos_out,
+                            dev.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return PC_ERR_CUDA;
   return PC_OK;
 }

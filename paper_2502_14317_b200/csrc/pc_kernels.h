@@ -21,6 +21,14 @@ cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m,
                                  int* idx, const float* calib, cudaStream_t st);
 cudaError_t launch_gather_kv(const void* k_src, const void* v_src, const long long stride_elems[3], const int* kept,
                              const int* idx, int m, int Hkv, int k, int d, void* k_out, void* v_out, int* pos_out,
-                             int sm_count, cudaStream_t st);
+                             int sm_count, bool by_slot, cudaStream_t st);
+
+// ---- pc_queue.cu (online chunk queue)
+void launch_queue_init(float* q_score, int* q_chunk, int m, cudaStream_t st);
+void launch_queue_update(const float* score, int Cb, int chunk_id0, int lower_is_better, int m, float* q_score,
+                         int* q_chunk, int* slot_src, cudaStream_t st);
+cudaError_t launch_queue_emit(const int* q_chunk, int m, int Hkv, int k, int d, const void* q_k, const void* q_v,
+                              const int* q_pos, int* kept_out, int* slot_order, void* k_out, void* v_out,
+                              int* pos_out, int sm_count, cudaStream_t st);
 
 }  // namespace pc

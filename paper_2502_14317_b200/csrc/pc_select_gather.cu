@@ -2,18 +2,9 @@
 // compressed-cache gather (Eq. 7, Eq. 9), and the single-layer stand-in for the chunk
 // self-information.  All HBM- or latency-bound; no tensor cores here on purpose.
 #include "pc_kernels.h"
+#include "pc_rank.cuh"
 
 namespace pc {
-
-// Monotone map float -> uint32 with "larger key = better".  NaN ranks worst, -0 == +0.
-__device__ __forceinline__ uint32_t rank_key(float f, bool lower_is_better) {
-  if (f != f) return 0u;
-  if (lower_is_better) f = -f;
-  uint32_t u = __float_as_uint(f);
-  if (u == 0x80000000u) u = 0u;                       // -0 -> +0
-  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-  return u == 0u ? 1u : u;                            // keep 0 for NaN only (-NaN patterns never reach here)
-}
 
 // ------------------------------------------------------------------ chunk score stand-in
 __global__ void chunk_score_kernel(const float* __restrict__ win_lse, int n_per_chunk, float* __restrict__ score) {
@@ -311,7 +302,9 @@ cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m,
 // ------------------------------------------------------------------ gather
 // One row of d bf16 (2d bytes) per (kv-head, slot); LPR lanes move one row with 16-byte
 // accesses, K and V in the same thread so both copies are in flight together.
-template <int D>
+// BY_SLOT (online chunk queue): kept[r] is the chunk that moves into slot r of the output, or -1 for a slot
+// that keeps its contents; the index rows are then those of the source chunk, idx[kept[r], hkv, :].
+template <int D, bool BY_SLOT>
 __global__ void __launch_bounds__(256) gather_kv_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src,
                                                         long long s_chunk, long long s_tok, long long s_head,   // in uint4 units
                                                         const int* __restrict__ kept, const int* __restrict__ idx, int m,
@@ -325,10 +318,12 @@ __global__ void __launch_bounds__(256) gather_kv_kernel(const uint4* __restrict_
     const int hk = (int)(row / ((long long)m * k));
     const int slot = (int)(row % ((long long)m * k));
     const int r = slot / k, t = slot % k;
-    const int j = idx[((size_t)r * Hkv + hk) * k + t];
+    const int c = kept[r];
+    if (BY_SLOT && c < 0) continue;
+    const int j = idx[((size_t)(BY_SLOT ? c : r) * Hkv + hk) * k + t];
     uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
     if (j >= 0) {
-      const long long off = (long long)kept[r] * s_chunk + (long long)j * s_tok + (long long)hk * s_head + sub;
+      const long long off = (long long)c * s_chunk + (long long)j * s_tok + (long long)hk * s_head + sub;
       kv = __ldg(k_src + off);
       vv = __ldg(v_src + off);
     }
@@ -340,19 +335,22 @@ __global__ void __launch_bounds__(256) gather_kv_kernel(const uint4* __restrict_
 
 cudaError_t launch_gather_kv(const void* k_src, const void* v_src, const long long stride_elems[3], const int* kept,
                              const int* idx, int m, int Hkv, int k, int d, void* k_out, void* v_out, int* pos_out,
-                             int sm_count, cudaStream_t st) {
+                             int sm_count, bool by_slot, cudaStream_t st) {
   const long long n_rows = (long long)Hkv * m * k;
   const int lpr = d / 8;
   long long want = (n_rows * lpr + 255) / 256;
   int blocks = (int)(want < (long long)sm_count * 8 ? want : (long long)sm_count * 8);
   if (blocks < 1) blocks = 1;
   const long long sc = stride_elems[0] / 8, stok = stride_elems[1] / 8, sh = stride_elems[2] / 8;
-  if (d == 128)
-    gather_kv_kernel<128><<<blocks, 256, 0, st>>>((const uint4*)k_src, (const uint4*)v_src, sc, stok, sh, kept, idx, m,
-                                                  Hkv, k, (uint4*)k_out, (uint4*)v_out, pos_out);
-  else
-    gather_kv_kernel<64><<<blocks, 256, 0, st>>>((const uint4*)k_src, (const uint4*)v_src, sc, stok, sh, kept, idx, m,
-                                                 Hkv, k, (uint4*)k_out, (uint4*)v_out, pos_out);
+#define PC_GATHER(D, S)                                                                                              \
+  gather_kv_kernel<D, S><<<blocks, 256, 0, st>>>((const uint4*)k_src, (const uint4*)v_src, sc, stok, sh, kept, idx, m, \
+                                                 Hkv, k, (uint4*)k_out, (uint4*)v_out, pos_out)
+  if (d == 128) {
+    if (by_slot) PC_GATHER(128, true); else PC_GATHER(128, false);
+  } else {
+    if (by_slot) PC_GATHER(64, true); else PC_GATHER(64, false);
+  }
+#undef PC_GATHER
   return cudaGetLastError();
 }
 

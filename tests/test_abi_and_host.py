@@ -70,6 +70,11 @@ def test_host_side_argument_errors_need_no_gpu(lib):
     assert lib.pc_gather_kv(p, p, None, 256, o, o, 2, 2, 64, 96, p, p, None, None) == -2   # head size
     assert lib.pc_parallel_attn(1, 24, 4, 2, 64, 128, p, 0, 1e4, 0.0, p, p, p, p, p, None, None, None, 0, None) == -2
     assert lib.pc_select_tokens_calibrated(p, o, 4, 2, 2, 256, 200, 64, -1, 0, 1.0, 1.0, 1.0, o, None) == -1   # n_s < 0
+    assert lib.pc_queue_init(0, p, o, None) == -1                    # no slots
+    assert lib.pc_queue_update(p, 4, -1, 1, 2, p, o, o, None) == -1  # negative chunk id
+    assert lib.pc_queue_update(p, 1000, 0, 1, 100, p, o, o, None) == -2   # slots + batch > 1024
+    assert lib.pc_queue_gather(p, p, None, 256, o, o, 2, 2, 64, 96, p, p, o, None) == -2   # head size
+    assert lib.pc_queue_emit(o, 2, 2, 64, 128, p, p, o, o, None, p, p, None, None) == -1    # no slot_order array
 
 
 def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
