@@ -338,6 +338,7 @@ def run_gpu(args, cfg):
         }
         if world == 1 and not args.no_extra:
             line["extra"] = extra_measurements(pc, torch, dev, peaks)
+            line["extra"]["streamed_hot_path"] = streamed_measurement(pc, torch, cfg, q, k, v, buffers)
         if not args.no_cpu_baseline and world == 1:
             v_cpu, s_cpu, desc = oracle_sample(cfg)
             line["cpu_baseline"] = {"value": v_cpu, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
@@ -359,6 +360,29 @@ def _time_us(torch, fn, warm=3, reps=20):
     e1.record()
     torch.cuda.synchronize()
     return 1e3 * e0.elapsed_time(e1) / reps
+
+
+def _tensor_bytes(torch, obj) -> int:
+    if isinstance(obj, torch.Tensor):
+        return obj.numel() * obj.element_size()
+    if isinstance(obj, dict):
+        return sum(_tensor_bytes(torch, x) for x in obj.values())
+    return 0
+
+
+def streamed_measurement(pc, torch, cfg, q, k, v, step_buffers, batch=4) -> dict:
+    """The same workload with the chunks taken `batch` at a time through the online chunk queue
+    (outside the timed region): time of one pass and the device memory held beyond the inputs."""
+    sb: dict = {}
+
+    def run():
+        pc.hot_path_streaming(q, k, v, w=cfg.w, rope_theta=cfg.rope_theta, m=cfg.m, k_keep=cfg.k, batch=batch, buffers=sb)
+    us = _time_us(torch, run, warm=2, reps=5)
+    tokens = cfg.C * cfg.L
+    return {"batch_chunks": batch, "ms": us / 1e3, "tokens_per_s": tokens / (us * 1e-6),
+            "intermediate_bytes": _tensor_bytes(torch, sb), "intermediate_bytes_all_chunks_at_once": _tensor_bytes(torch, step_buffers),
+            "note": "pc_chunk_prefill_attn + pc_select_tokens on every chunk + pc_queue_update/gather per batch, "
+                    "pc_queue_emit + pc_parallel_attn at the end; same results as the timed step"}
 
 
 def extra_measurements(pc, torch, dev, peaks, only=None, select_chunks=8192) -> dict:
