@@ -386,55 +386,80 @@ def hot_path(q, k, v, *, w, rope_theta, m, k_keep, softmax_scale=0.0, chunk_scor
     return res
 
 
-def hot_path_streaming(q, k, v, *, w, rope_theta, m, k_keep, batch, softmax_scale=0.0, chunk_score=None, buffers=None):
-    """The whole path with the chunks taken ``batch`` at a time through the online chunk queue.
+def hot_path_streaming(q, k, v, *, w, rope_theta, m, k_keep, batch=None, softmax_scale=0.0, chunk_score=None,
+                       buffers=None):
+    """The whole path with the chunks taken one batch at a time through the online chunk queue.
 
     Per batch: chunk-local attention, token eviction on EVERY chunk of the batch, queue update, and the
     compressed caches of the chunks that entered the queue are copied into their slots; the batch's outputs
     (attention output, rotated keys, window scores) live in buffers of batch size that the next batch
     overwrites, so device memory beyond the inputs is O(batch + m) chunks whatever C is.  After the last batch
     the queue is emitted in chunk order and the window attends over it.  Same results as :func:`hot_path`
-    (kept chunks, indices and compressed cache bit for bit).  q, k, v here are whole device tensors
-    [C,L,*,d]; a caller that streams from elsewhere makes the same calls on its own batches.
+    (kept chunks, indices and compressed cache bit for bit).
+
+    q, k, v are either whole device tensors [C,L,*,d], cut into batches of ``batch`` chunks, or lists of
+    per-batch tensors [Cb,L_b,*,d].  In a list the chunk length may differ from batch to batch (a shorter
+    last chunk is a batch of its own: its window directly follows its context, and only the k_keep tokens it
+    contributes persist); every L_b - w must be at least k_keep.  The query window of the global attention is
+    taken from the first chunk of the first batch.  A caller that streams from elsewhere makes the same calls
+    on its own batches.
     """
     b = {} if buffers is None else buffers
-    C, L, Hq, d = q.shape
-    Hkv = k.shape[2]
-    dev = q.device
+    if isinstance(q, (list, tuple)):
+        batches = list(zip(q, k, v))
+    else:
+        if batch is None:
+            raise PcError("hot_path_streaming needs a batch size for whole tensors")
+        batches = [(q[c0:c0 + batch], k[c0:c0 + batch], v[c0:c0 + batch]) for c0 in range(0, q.shape[0], batch)]
+    q0, k0, v0 = batches[0]
+    _, L0, Hq, d = q0.shape
+    Hkv = k0.shape[2]
+    dev = q0.device
+    n_max = max(bq.shape[0] for bq, _, _ in batches)
     if "queue" not in b:
         b["queue"] = queue_init(m, Hkv, k_keep, d, dev)
-        b["ids"] = torch.arange(batch, dtype=torch.int32, device=dev)
     else:
         lib = load_library()
         _check(lib.pc_queue_init(m, _ptr(b["queue"]["q_score"]), _ptr(b["queue"]["q_chunk"]), _stream()), "pc_queue_init")
+    if "ids" not in b or b["ids"].numel() < n_max:
+        b["ids"] = torch.arange(n_max, dtype=torch.int32, device=dev)
     qu = b["queue"]
-    pre = None
-    for c0 in range(0, C, batch):
-        c1 = min(c0 + batch, C)
-        n = c1 - c0
-        tag = "full" if n == batch else "tail"                 # a shorter last batch has buffers of its own
-        pb = b.setdefault("pre_" + tag, {})
-        pre = chunk_prefill_attn(q[c0:c1], k[c0:c1], v[c0:c1], w=w, rope_theta=rope_theta, softmax_scale=softmax_scale,
+    c0 = 0
+    k_win = None
+    for bq, bk, bv in batches:
+        n, L = bq.shape[0], bq.shape[1]
+        if L - w < k_keep:
+            raise PcError("a chunk of %d tokens has fewer than k_keep = %d context tokens" % (L, k_keep))
+        pb = b.setdefault("pre_%dx%d" % (n, L), {})            # buffers per batch shape
+        pre = chunk_prefill_attn(bq, bk, bv, w=w, rope_theta=rope_theta, softmax_scale=softmax_scale,
                                  out=pb.get("o"), k_rot=pb.get("k_rot"), win_score=pb.get("win_score"),
                                  win_lse=pb.get("win_lse"), status=b.get("status"), workspace=pb.get("workspace"))
         b["status"] = pre["status"]
         pb.update({"o": pre["o"], "k_rot": pre["k_rot"], "win_score": pre["win_score"], "win_lse": pre["win_lse"],
                    "workspace": pre["workspace"]})
-        score = chunk_score[c0:c1] if chunk_score is not None else chunk_score_from_lse(pre["win_lse"], out=pb.get("score"))
-        pb["score"] = score if chunk_score is None else pb.get("score")
+        if chunk_score is not None:
+            score = chunk_score[c0:c0 + n]
+        else:
+            score = chunk_score_from_lse(pre["win_lse"], out=pb.get("score"))
+            pb["score"] = score
         idx = select_tokens(pre["win_score"], b["ids"][:n], L - w, k_keep, out=pb.get("idx"))
         pb["idx"] = idx
         queue_update(qu, score, c0, True)
-        queue_gather(qu, pre["k_rot"], v[c0:c1], idx)
+        queue_gather(qu, pre["k_rot"], bv, idx)
+        if k_win is None:                                      # the window is the same in every chunk: keep the first
+            k_win = b.get("k_win")
+            if k_win is None or k_win.shape != (1, w, Hkv, d):
+                k_win = torch.empty((1, w, Hkv, d), dtype=torch.bfloat16, device=dev)
+            k_win.copy_(pre["k_rot"][0:1, L - w:])
+            b["k_win"] = k_win
+        c0 += n
     kept, kc, vc, pos = queue_emit(qu, k_out=b.get("kc"), v_out=b.get("vc"), pos_out=b.get("pos"), kept_out=b.get("kept"))
     b.update({"kc": kc, "vc": vc, "pos": pos, "kept": kept})
-    q_win = q[0:1, L - w:]
+    q_win = q0[0:1, L0 - w:]
     q_win = q_win if q_win.is_contiguous() else q_win.contiguous()
-    k_win = pre["k_rot"][0:1, L - w:]                           # the window is the same in every chunk
-    k_win = k_win if k_win.is_contiguous() else k_win.contiguous()
-    v_win = v[0:1, L - w:]
+    v_win = v0[0:1, L0 - w:]
     v_win = v_win if v_win.is_contiguous() else v_win.contiguous()
-    pa = parallel_attn(q_win, kc.unsqueeze(0), vc.unsqueeze(0), k_win, v_win, q_pos0=L - w, rope_theta=rope_theta,
+    pa = parallel_attn(q_win, kc.unsqueeze(0), vc.unsqueeze(0), k_win, v_win, q_pos0=L0 - w, rope_theta=rope_theta,
                        softmax_scale=softmax_scale, out=b.get("fg"), status=b["status"], workspace=b.get("ws_par"))
     b.update({"fg": pa["out"], "ws_par": pa["workspace"]})
     return {"kept": kept, "kc": kc, "vc": vc, "pos": pos, "fg": pa["out"], "status": b["status"]}

@@ -138,3 +138,65 @@ def test_streaming_path_cfg1_batches_of_4():
     rng = np.random.default_rng(7)
     # scores that make every batch change the queue
     _check_streaming(cfg, inp, 4, chunk_score=rng.permutation(cfg.C).astype(np.float32), check_fg=True)
+
+
+def test_streaming_with_a_shorter_last_chunk(cfg0_inputs):
+    """An input whose length is not a multiple of the chunk length: three chunks of 256 tokens and a last one of
+    200 (window included).  The short chunk is a batch of its own; its window sits right behind its context, at
+    positions 184..199.  The oracle is composed per chunk length from the same pinned pieces."""
+    import dataclasses
+    import paper_2502_14317_b200 as pc
+    cfg, inp = cfg0_inputs
+    w, m, kk, theta = cfg.w, 2, cfg.k, cfg.rope_theta
+    La, Lb = cfg.L, 200
+    scale = 1.0 / np.sqrt(cfg.d)
+    cfg_b = dataclasses.replace(cfg, name="tail", C=1, L=Lb, n_planted_chunks=0, seed=cfg.seed + 77, planted_chunks=())
+    tail = pc_inputs.make_prefill_inputs(cfg_b)
+    qa, ka, va = inp["q"][:3], inp["k"][:3], inp["v"][:3]
+    qb, kb, vb = tail["q"].copy(), tail["k"].copy(), tail["v"].copy()
+    qb[:, Lb - w:], kb[:, Lb - w:], vb[:, Lb - w:] = qa[:1, La - w:], ka[:1, La - w:], va[:1, La - w:]   # same query tokens
+    host = [(qa, ka, va), (qb, kb, vb)]
+    dev = [tuple(to_dev(t) for t in b) for b in host]
+
+    # per-batch tensors of the CUDA path, checked against the oracle, then ranked by the oracle as they are
+    S_all, krot_all, score_all = [], [], []
+    for (q, k, v), (dq, dk, dv) in zip(host, dev):
+        L = q.shape[1]
+        pre = pc.chunk_prefill_attn(dq, dk, dv, w=w, rope_theta=theta)
+        sc = pc.chunk_score_from_lse(pre["win_lse"])
+        torch.cuda.synchronize()
+        assert int(pre["status"].item()) == 0
+        q_rot, k_rot = orc.rope_bf16(q, theta), orc.rope_bf16(k, theta)
+        assert np.array_equal(to_bits(pre["k_rot"]), k_rot)
+        S, _, LSE_win = orc.window_scores(q_rot, k_rot, v, w, scale)
+        S_gpu = pre["win_score"].cpu().numpy()
+        d = np.abs(S_gpu - S)
+        assert np.all(d <= 1e-3 * np.maximum(S, cfg.G * w / L))
+        assert np.allclose(sc.cpu().numpy(), orc.chunk_score_from_lse(LSE_win), atol=2e-3)
+        S_all.append(S_gpu)
+        krot_all.append(k_rot)
+        score_all.append(sc.cpu().numpy())
+
+    for forced in (None, np.array([3.0, 1.0, 4.0, 0.5], dtype=np.float32)):     # second case: the short chunk is kept
+        score = np.concatenate(score_all) if forced is None else forced
+        kept_o = orc.select_chunks(score, m)
+        Kc_o, Vc_o, pos_o = [], [], []
+        for c in kept_o:
+            bi, local = (0, int(c)) if c < 3 else (1, 0)
+            n_cand = host[bi][0].shape[1] - w
+            idx = orc.select_tokens(S_all[bi], np.array([local]), n_cand, kk)
+            K1, V1, P1 = orc.gather_kv(krot_all[bi], host[bi][2], np.array([local]), idx)
+            Kc_o.append(K1); Vc_o.append(V1); pos_o.append(P1)
+        Kc_o, Vc_o, pos_o = (np.concatenate(x, axis=1) for x in (Kc_o, Vc_o, pos_o))
+        got = pc.hot_path_streaming([b[0] for b in dev], [b[1] for b in dev], [b[2] for b in dev], w=w, rope_theta=theta,
+                                    m=m, k_keep=kk, chunk_score=None if forced is None else torch.from_numpy(forced).cuda())
+        torch.cuda.synchronize()
+        assert int(got["status"].item()) == 0
+        assert np.array_equal(got["kept"].cpu().numpy(), kept_o)
+        assert np.array_equal(got["pos"].cpu().numpy(), pos_o)
+        assert np.array_equal(to_bits(got["kc"]), Kc_o) and np.array_equal(to_bits(got["vc"]), Vc_o)
+        Fg, _ = orc.parallel_attention(qa[0:1, La - w:], La - w, theta, None, Kc_o[None], Vc_o[None],
+                                       krot_all[0][0:1, La - w:], va[0:1, La - w:])
+        check_attention_output(to_f64(got["fg"]), Fg, "Fg (ragged)")
+    if forced is not None:
+        assert 3 in kept_o.tolist()
