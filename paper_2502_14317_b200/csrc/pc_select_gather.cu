@@ -122,11 +122,19 @@ __device__ __forceinline__ int sel_ordered_offsets(uint32_t x, int lane, int war
   return total;
 }
 
-template <bool CAL>
+// One thread adds to a counter in shared memory (the compiler is not asked to aggregate over the warp again).
+__device__ __forceinline__ void sel_red_add(int* p, int v) {
+  asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(p))), "r"(v) : "memory");
+}
+
+// STAGE: the kept positions are first put in order in shared memory (k words) and written out coalesced;
+// otherwise (k too large for that) they are stored straight to the index row.
+template <bool CAL, bool STAGE>
 __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const float* __restrict__ win_score,
                                                                         const int* __restrict__ kept, int Hkv, int L,
                                                                         int n_cand, int k, int* __restrict__ idx,
                                                                         const SelCalib cal) {
+  extern __shared__ int sel_stage[];                           // STAGE: [min(k, n_cand)]
   __shared__ int s_cnt[32];                                    // per bit: undecided keys of the row with that bit set
   __shared__ int s_tot[2][32];
 
@@ -237,7 +245,7 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
     const uint32_t slice = bit == 31 ? ~neg : key[31 - bit] ^ neg;   // this bit of the order-preserving images
     const uint32_t ones = active & slice;
     const int cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(ones));
-    if (lane == 0) atomicAdd(&s_cnt[bit], cnt);
+    if (lane == 0) sel_red_add(&s_cnt[bit], cnt);
     __syncthreads();
     const int tot = s_cnt[bit];                                // undecided keys with this bit set
     if (tot >= need) {                                         // the k-th largest has this bit
@@ -274,13 +282,31 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
   }
   int offs[8];
   const int n_emit = sel_ordered_offsets(taken, lane, warp, nwarps, s_tot[0], offs);
+  if (STAGE) {
+    const uint32_t stage_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(sel_stage));
 #pragma unroll
-  for (int i = 0; i < SEL_KPT; ++i) {
-    const bool t = (taken & (0x80000000u >> i)) != 0u;
-    if (t) out[offs[i >> 2]] = pbase + 128 * (i >> 2) + (i & 3);
-    offs[i >> 2] += t ? 1 : 0;
+    for (int j = 0; j < 8; ++j) {
+      uint32_t addr = stage_u32 + 4u * offs[j];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {                            // predicated store and advance: no branch per key
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %1, 0;\n\t@p st.shared.u32 [%0], %2;\n\t@p add.u32 %0, %0, 4;\n\t}"
+            : "+r"(addr)
+            : "r"(taken & (0x80000000u >> (4 * j + e))), "r"(pbase + 128 * j + e)
+            : "memory");
+      }
+    }
+    __syncthreads();
+    for (int j = tid; j < k_out; j += blockDim.x) out[j] = j < n_emit ? sel_stage[j] : -1;
+  } else {
+#pragma unroll
+    for (int i = 0; i < SEL_KPT; ++i) {
+      const bool t = (taken & (0x80000000u >> i)) != 0u;
+      if (t) out[offs[i >> 2]] = pbase + 128 * (i >> 2) + (i & 3);
+      offs[i >> 2] += t ? 1 : 0;
+    }
+    for (int j = n_emit + tid; j < k_out; j += blockDim.x) out[j] = -1;
   }
-  for (int j = n_emit + tid; j < k_out; j += blockDim.x) out[j] = -1;
 }
 
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
@@ -289,13 +315,19 @@ cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m,
   int threads = (n_cand + SEL_SPAN - 1) / SEL_SPAN * 32;
   if (threads < 32) threads = 32;
   if (threads > SEL_MAX_THREADS) return cudaErrorInvalidValue;
+  const SelCalib cal = calib ? SelCalib{1, (int)calib[0], (int)calib[1], calib[2], calib[3], calib[4]}
+                             : SelCalib{0, 0, 0, 0.f, 0.f, 0.f};
+  const size_t stage_bytes = sizeof(int) * (size_t)(k < n_cand ? k : n_cand);
+  const bool stage = stage_bytes <= 40 * 1024;                 // within the default dynamic shared-memory limit
+  const int grid = m * Hkv;
+#define PC_SELECT(C, S) \
+  select_tokens_kernel<C, S><<<grid, threads, S ? stage_bytes : 0, st>>>(win_score, kept, Hkv, L, n_cand, k, idx, cal)
   if (calib) {
-    const SelCalib cal{1, (int)calib[0], (int)calib[1], calib[2], calib[3], calib[4]};
-    select_tokens_kernel<true><<<m * Hkv, threads, 0, st>>>(win_score, kept, Hkv, L, n_cand, k, idx, cal);
+    if (stage) PC_SELECT(true, true); else PC_SELECT(true, false);
   } else {
-    const SelCalib cal{0, 0, 0, 0.f, 0.f, 0.f};
-    select_tokens_kernel<false><<<m * Hkv, threads, 0, st>>>(win_score, kept, Hkv, L, n_cand, k, idx, cal);
+    if (stage) PC_SELECT(false, true); else PC_SELECT(false, false);
   }
+#undef PC_SELECT
   return cudaGetLastError();
 }
 

@@ -50,6 +50,8 @@ def test_chunk_score_from_lse():
     (2, 2, 300, 16, 284, 2),         # k = n_cand: identity
     (1, 2, 100, 4, 120, 1),          # k > n_cand: padding with -1
     (1, 1, 32768, 8, 5000, 1),       # largest supported row
+    (2, 2, 20000, 64, 12000, 2),     # k too large for the staged output: direct ordered stores
+    (1, 1, 32768, 8, 32000, 1),      # the same at the largest row
 ])
 def test_select_tokens(C, Hkv, L, w, k, m):
     import paper_2502_14317_b200 as pc
@@ -111,6 +113,7 @@ def test_keep_all_gather_is_a_reshape():
     (2, 1, 8192, 64, 2048, 8, 100, 100, (float("inf"), 0.97, float("inf"))),   # workload row shape, middle peaks only
     (1, 1, 200, 8, 50, 1, 150, 150, (0.2, 0.3, 0.4)),           # overlapping regions: the sink region wins
     (2, 2, 400, 8, 30, 2, 100, 100, (0.0, 0.0, 0.0)),           # everything above the thresholds: all -1
+    (1, 1, 16000, 64, 11000, 2, 100, 100, (0.9, 0.95, 0.9)),    # k too large for the staged output
 ])
 def test_select_tokens_calibrated(C, m, L, w, k, Hkv, n_s, n_r, lams):
     import paper_2502_14317_b200 as pc
