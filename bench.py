@@ -275,7 +275,7 @@ def run_gpu(args, cfg):
         # public API for host inputs: uploads the chunks in groups on a copy stream while the attention of the
         # previous group runs; every byte of Q, K, V crosses PCIe inside the timed region, and the result comes back
         res = pc.hot_path_from_host(hq, hk, hv, w=w, rope_theta=cfg.rope_theta, m=cfg.m, k_keep=cfg.k,
-                                    n_groups=min(4, cfg.C), buffers=e2e_buffers)
+                                    n_groups=min(16, cfg.C), buffers=e2e_buffers)
         h_out.copy_(res["fg"], non_blocking=True)
 
     e2e_step()
