@@ -47,13 +47,14 @@ void fill_strides(const int64_t in[3], int64_t out[3], int64_t tokens, int64_t h
 bool strides_ok(const int64_t s[3], int64_t d) { return s[0] > 0 && s[1] > 0 && s[2] >= d && s[0] % 8 == 0 && s[1] % 8 == 0 && s[2] % 8 == 0; }
 
 struct PrefillLayout {
-  size_t off_counter, off_table, off_krot, total;
+  size_t off_counter, off_table, off_table32, off_krot, total;
 };
 PrefillLayout prefill_layout(const pc_prefill_desc* d, bool krot_in_ws) {
   PrefillLayout l;
   size_t off = 0;
   l.off_counter = off; off += ALIGN;
   l.off_table = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(double2));
+  l.off_table32 = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(float2));
   l.off_krot = off;
   if (krot_in_ws) off += align_up((size_t)d->C * d->L * d->Hkv * d->d * 2);
   l.total = off;
@@ -121,6 +122,7 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   int* counter = reinterpret_cast<int*>(ws + lay.off_counter);
   double2* table = reinterpret_cast<double2*>(ws + lay.off_table);
+  float2* table32 = reinterpret_cast<float2*>(ws + lay.off_table32);
   void* krot = krot_in_ws ? static_cast<void*>(ws + lay.off_krot) : k_rot;
 
   // tensor maps (innermost first: d, head, token, chunk)
@@ -143,7 +145,7 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
     return PC_ERR_CUDA;
 
   if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return PC_ERR_CUDA;
-  pc::launch_rope_table(table, desc->L, d, (double)desc->rope_theta, 0, st);
+  pc::launch_rope_table(table, table32, desc->L, d, (double)desc->rope_theta, 0, st);
   const long long ks_ll[3] = {ks[0], ks[1], ks[2]};
   pc::launch_rope_keys(k, ks_ll, krot, table, desc->C, desc->L, desc->Hkv, d, st);
 
@@ -152,6 +154,7 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
   const double scale = desc->softmax_scale > 0.0f ? (double)desc->softmax_scale : 1.0 / std::sqrt((double)d);
   prm.scale_log2 = (float)(scale * 1.4426950408889634);
   prm.rope_tab = table;
+  prm.rope_tab32 = table32;
   prm.lse = lse; prm.win_lse = win_lse; prm.win_score = win_score;
   prm.status = status_word; prm.counter = counter;
   // head size 128 runs on CTA pairs (cta_group::2); head size 64 on single CTAs with two blocks
@@ -385,7 +388,7 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
     return PC_ERR_CUDA;
 
   if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return PC_ERR_CUDA;
-  pc::launch_rope_table(table, w, d, (double)rope_theta, q_pos0, st);
+  pc::launch_rope_table(table, nullptr, w, d, (double)rope_theta, q_pos0, st);
 
   pc::ParallelParams prm;
   prm.B = B; prm.w = w; prm.Hq = Hq; prm.Hkv = Hkv; prm.Nk = Nk;

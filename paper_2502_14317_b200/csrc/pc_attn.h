@@ -11,6 +11,7 @@ struct PrefillParams {
   int C, L, w, Hq, Hkv;
   float scale_log2;              // softmax scale * log2(e)
   const double2* rope_tab;       // [L][d/2] (cos, sin)
+  const float2* rope_tab32;      // the same table rounded to fp32
   float* lse;                    // [C,Hq,L] or null
   float* win_lse;                // [C,Hq,w]
   float* win_score;              // [C,Hkv,L]

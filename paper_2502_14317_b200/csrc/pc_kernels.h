@@ -7,8 +7,9 @@
 namespace pc {
 
 // ---- pc_rope.cu
-// cos/sin table: tab[p * (d/2) + t] = (cos, sin)(  (pos0 + p) * theta^(-2t/d) ), fp64.
-void launch_rope_table(double2* tab, int n_pos, int d, double theta, int pos0, cudaStream_t st);
+// cos/sin table: tab[p * (d/2) + t] = (cos, sin)(  (pos0 + p) * theta^(-2t/d) ), fp64; tab32 (may be null): the
+// same entries rounded to fp32.
+void launch_rope_table(double2* tab, float2* tab32, int n_pos, int d, double theta, int pos0, cudaStream_t st);
 // k_rot[c,p,h,:] = bf16( RoPE(k[c,p,h,:], position p) ), rotation evaluated in fp64.
 void launch_rope_keys(const void* k, const long long k_stride[3], void* k_rot, const double2* tab, int C, int L,
                       int Hkv, int d, cudaStream_t st);

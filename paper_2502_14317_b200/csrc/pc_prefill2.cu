@@ -32,7 +32,7 @@
 #define PC2_EARLY_ROT 1
 #endif
 #ifndef PC2_POLY_PAIRS_PER_8
-#define PC2_POLY_PAIRS_PER_8 2
+#define PC2_POLY_PAIRS_PER_8 0
 #endif
 
 namespace pc {
@@ -169,34 +169,60 @@ __device__ __forceinline__ void mbar_wait_cluster(uint64_t* bar, uint32_t parity
   }
 }
 
-// RoPE of half of row `row` of a 128-byte-swizzled [128 x 128] bf16 Q tile (two atoms of 64 columns):
-// pairs (t, t + 64) for t in [32 * part, 32 * part + 32) at position `pos`; fp64, one rounding.
-__device__ __forceinline__ void rope_row_part(uint8_t* tile, int row, int part, int pos, const double2* __restrict__ tab) {
-  const double2* tab_row = tab + (size_t)pos * (D / 2);
-#pragma unroll 2
-  for (int cidx = part * 4; cidx < part * 4 + 4; ++cidx) {
-    uint8_t* lo_p = tile + sw128_offset(row, cidx);
-    uint8_t* hi_p = tile + 16384 + sw128_offset(row, cidx);
-    const uint4 lo = *reinterpret_cast<const uint4*>(lo_p);
-    const uint4 hi = *reinterpret_cast<const uint4*>(hi_p);
-    const uint32_t lo_w[4] = {lo.x, lo.y, lo.z, lo.w}, hi_w[4] = {hi.x, hi.y, hi.z, hi.w};
-    uint32_t out_lo[4], out_hi[4];
+// RoPE of 16 rows of a 128-byte-swizzled [128 x 128] bf16 Q tile (two atoms of 64 columns) by one warp:
+// rows row0 .. row0 + 15, row i at position pos_of(i) (negative: leave the row alone).  Lane l takes the
+// pairs (t, t + 64) for t = 2l, 2l + 1 of a row, so a warp reads a row of the cos/sin table as one
+// contiguous block (with a thread per row every lane reads its own table row: 32 cache lines per load
+// instruction), and the table reads of all 16 rows are in flight together.
+// The result is the fp64 rotation rounded once to bf16, bit for bit, but fp64 arithmetic (and the
+// fp32 <-> fp64 conversions around it, which run at a fraction of the fp32 rate) is only used where it
+// matters: the rotation is first evaluated in fp32 with the fp32 copy of the table; its error is below
+// 2^-22 (|x1| + |x2|), so when y - tol and y + tol with tol = 2^-21 (|x1| + |x2|) round to the same bf16
+// value, that value is the correctly rounded one.  Otherwise (about one output in a few thousand) the
+// pair is redone in fp64.
+template <typename PosOf>
+__device__ __forceinline__ void rope_rows_warp(uint8_t* tile, int row0, int lane, const double2* __restrict__ tab,
+                                               const float2* __restrict__ tab32, PosOf pos_of) {
+  // all reads first, then the arithmetic, then all writes: reads and writes of the tile go through
+  // pointers the compiler cannot tell apart, so a write in the middle would serialise the rows
+  float4 cs[16];
+  uint32_t lo[16], hi[16];
+  int pos[16];
+  uint8_t* const lo_base = tile + (lane & 3) * 4;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint32_t rl = 0, rh = 0;
+  for (int i = 0; i < 16; ++i) {
+    pos[i] = pos_of(row0 + i);
+    cs[i] = __ldg(reinterpret_cast<const float4*>(tab32 + (size_t)(pos[i] < 0 ? 0 : pos[i]) * (D / 2) + 2 * lane));
+    const uint8_t* lo_p = lo_base + sw128_offset(row0 + i, lane >> 2);
+    lo[i] = *reinterpret_cast<const uint32_t*>(lo_p);
+    hi[i] = *reinterpret_cast<const uint32_t*>(lo_p + 16384);
+  }
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const double x1 = (double)__uint_as_float(((lo_w[i] >> (16 * e)) & 0xFFFFu) << 16);
-        const double x2 = (double)__uint_as_float(((hi_w[i] >> (16 * e)) & 0xFFFFu) << 16);
-        const double2 t = tab_row[cidx * 8 + 2 * i + e];
-        rl |= (uint32_t)f64_to_bf16_rne(x1 * t.x - x2 * t.y) << (16 * e);
-        rh |= (uint32_t)f64_to_bf16_rne(x2 * t.x + x1 * t.y) << (16 * e);
-      }
-      out_lo[i] = rl;
-      out_hi[i] = rh;
+  for (int i = 0; i < 16; ++i) {
+    const float a0 = __uint_as_float(lo[i] << 16), a1 = __uint_as_float(lo[i] & 0xFFFF0000u);   // x1 of pairs 2l, 2l + 1
+    const float b0 = __uint_as_float(hi[i] << 16), b1 = __uint_as_float(hi[i] & 0xFFFF0000u);   // x2
+    const float c0 = cs[i].x, s0 = cs[i].y, c1 = cs[i].z, s1 = cs[i].w;
+    const float yl0 = fmaf(-b0, s0, a0 * c0), yh0 = fmaf(a0, s0, b0 * c0);
+    const float yl1 = fmaf(-b1, s1, a1 * c1), yh1 = fmaf(a1, s1, b1 * c1);
+    const float tol0 = 4.76837158203125e-7f * (fabsf(a0) + fabsf(b0)), tol1 = 4.76837158203125e-7f * (fabsf(a1) + fabsf(b1));
+    uint32_t rl = pack_bf16x2(yl0 - tol0, yl1 - tol1), rh = pack_bf16x2(yh0 - tol0, yh1 - tol1);
+    const uint32_t rl_up = pack_bf16x2(yl0 + tol0, yl1 + tol1), rh_up = pack_bf16x2(yh0 + tol0, yh1 + tol1);
+    if ((rl != rl_up || rh != rh_up) && pos[i] >= 0) {         // too close to a rounding boundary: exact
+      const double2* tab_row = tab + (size_t)pos[i] * (D / 2) + 2 * lane;
+      const double2 t0 = __ldg(tab_row), t1 = __ldg(tab_row + 1);
+      const double da0 = (double)a0, da1 = (double)a1, db0 = (double)b0, db1 = (double)b1;
+      rl = (uint32_t)f64_to_bf16_rne(da0 * t0.x - db0 * t0.y) | ((uint32_t)f64_to_bf16_rne(da1 * t1.x - db1 * t1.y) << 16);
+      rh = (uint32_t)f64_to_bf16_rne(db0 * t0.x + da0 * t0.y) | ((uint32_t)f64_to_bf16_rne(db1 * t1.x + da1 * t1.y) << 16);
     }
-    *reinterpret_cast<uint4*>(lo_p) = make_uint4(out_lo[0], out_lo[1], out_lo[2], out_lo[3]);
-    *reinterpret_cast<uint4*>(hi_p) = make_uint4(out_hi[0], out_hi[1], out_hi[2], out_hi[3]);
+    lo[i] = rl;
+    hi[i] = rh;
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    if (pos[i] < 0) continue;
+    uint8_t* lo_p = lo_base + sw128_offset(row0 + i, lane >> 2);
+    *reinterpret_cast<uint32_t*>(lo_p) = lo[i];
+    *reinterpret_cast<uint32_t*>(lo_p + 16384) = hi[i];
   }
 }
 
@@ -478,10 +504,13 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     bool pre_rotated = false;                                // the next block's Q is already rotated (cQ counts it)
     auto rotate_q = [&](const Blk& b) {                      // RoPE of a Q tile in shared memory, half a row per thread
       const int qb = cQ & 1;
-      const int tok = b.t * TILE + r;
       WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
       ++cQ;
-      if (tok < prm.L) rope_row_part(cx.sQ[qb], r, hlf, tok, prm.rope_tab);
+      {
+        const int tok0 = b.t * TILE, L = prm.L;
+        rope_rows_warp(cx.sQ[qb], warp * 16, lane, prm.rope_tab, prm.rope_tab32,
+                       [=](int row) { return tok0 + row < L ? tok0 + row : -1; });
+      }
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.q_ready[qb], 0));
@@ -702,7 +731,11 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int qb = cQ & 1;
           WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
           ++cQ;
-          if (r < rows_half) rope_row_part(cx.sQ[qb], r, hlf, prm.L - prm.w + (r % prm.w), prm.rope_tab);
+          {
+            const int w0 = prm.L - prm.w, ww = prm.w, nr = rows_half;
+            rope_rows_warp(cx.sQ[qb], warp * 16, lane, prm.rope_tab, prm.rope_tab32,
+                           [=](int row) { return row < nr ? w0 + (row % ww) : -1; });
+          }
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.q_ready[qb], 0));

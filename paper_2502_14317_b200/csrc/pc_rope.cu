@@ -6,7 +6,8 @@
 
 namespace pc {
 
-__global__ void rope_table_kernel(double2* __restrict__ tab, int n_pos, int half, double theta, int pos0) {
+__global__ void rope_table_kernel(double2* __restrict__ tab, float2* __restrict__ tab32, int n_pos, int half, double theta,
+                                  int pos0) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_pos * half) return;
   const int p = i / half, t = i % half;
@@ -15,11 +16,12 @@ __global__ void rope_table_kernel(double2* __restrict__ tab, int n_pos, int half
   double s, c;
   sincos(phi, &s, &c);
   tab[i] = make_double2(c, s);
+  if (tab32 != nullptr) tab32[i] = make_float2((float)c, (float)s);   // the same entries rounded to fp32
 }
 
-void launch_rope_table(double2* tab, int n_pos, int d, double theta, int pos0, cudaStream_t st) {
+void launch_rope_table(double2* tab, float2* tab32, int n_pos, int d, double theta, int pos0, cudaStream_t st) {
   const int n = n_pos * (d / 2);
-  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, n_pos, d / 2, theta, pos0);
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, tab32, n_pos, d / 2, theta, pos0);
 }
 
 // One thread owns 8 consecutive pairs (t..t+7) of one position and walks all heads and a
