@@ -49,7 +49,7 @@ def test_workspace_queries_are_host_only(lib):
     assert binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128) == 256 + 8192 * 64 * 16 + 8192 * 64 * 8
     assert binding.chunk_prefill_attn_workspace_bytes(4, 256, 16, 4, 2, 64) == 256 + 256 * 32 * 16 + 256 * 32 * 8
     with_krot = binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128, k_rot_in_workspace=True)
-    assert with_krot == 256 + 8192 * 64 * 16 + 16 * 8192 * 8 * 128 * 2
+    assert with_krot == 256 + 8192 * 64 * 16 + 8192 * 64 * 8 + 16 * 8192 * 8 * 128 * 2
     # unsupported shapes give 0
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 24, 4, 2, 64) == 0       # window not a power of two
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 2, 96) == 0       # head size
