@@ -15,7 +15,10 @@
 namespace pc {
 
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // ~1 s at B200 clocks
-constexpr unsigned SPIN_BACKOFF_NS = 40;                // pause between two polls of a barrier
+#ifndef PC_SPIN_BACKOFF_NS
+#define PC_SPIN_BACKOFF_NS 20
+#endif
+constexpr unsigned SPIN_BACKOFF_NS = PC_SPIN_BACKOFF_NS;   // pause between two polls of a barrier (0: none)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -57,7 +60,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    __nanosleep(SPIN_BACKOFF_NS);             // a hot spin takes issue slots from the warps that share the scheduler
+    if (SPIN_BACKOFF_NS > 0) __nanosleep(SPIN_BACKOFF_NS);   // a hot spin takes issue slots from the warps that share the scheduler
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
