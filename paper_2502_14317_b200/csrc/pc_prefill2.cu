@@ -8,11 +8,12 @@
 // and the tensor cores of both SMs read both halves.  That halves the shared-memory traffic
 // per MMA, which is what limits a single CTA with two blocks at this head size.
 //
-// Per CTA, TMEM holds three S/P buffers (3 x 128 columns) and one accumulator (128 columns).
-// With three S buffers Q K^T of tile j+1, j+2 does not wait for the softmax of tile j: the
-// pipe runs  S(j+2) = Q K^T  and  O += P(j) V  while two softmax warpgroups turn S(j+1), S(j+2)
-// into P: they take alternate key tiles (thread = query row), chained only through the short
-// per-row decision on the running maximum, so the MUFU pipe always has exponentials to do.
+// Per CTA, TMEM holds two S buffers (one per softmax warpgroup, 128 columns each), two P buffers
+// (64 columns of bf16 each) and one accumulator (128 columns).  Two softmax warpgroups take
+// alternate key tiles (thread = query row), chained only through the short per-row decision on the
+// running maximum.  As soon as a warpgroup has S(j) in registers, Q K^T of its next tile S(j+2)
+// may run into the same buffer, so that S is waiting when the warpgroup comes back; P(j) goes to
+// the warpgroup's P buffer once P V of its previous tile has run.
 //
 // Warps (12 per CTA): 0-3 softmax of even tiles, 4-7 softmax of odd tiles (both: Q rotation,
 // epilogue and score sweep split by halves),
@@ -44,7 +45,8 @@ constexpr int D = 128;
 constexpr int NT2 = 384;                     // threads per CTA
 constexpr int WARP_PRODUCER = 8, WARP_QK = 9, WARP_PV = 10;
 constexpr int NKS = 4, NVS = 4;              // K / V ring stages (16 KB each)
-constexpr int NSB = 3;                       // S/P buffers in TMEM
+constexpr int NSB = 2;                       // S buffers in TMEM (one per warpgroup); P has buffers of its own
+constexpr uint32_t TM_P = 256;               // two P buffers of 64 columns (128 bf16 keys each), one per warpgroup
 constexpr int HALF_BYTES = 16384;            // 64 keys x 128 d of K, or 128 keys x 64 d of V
 constexpr int Q_BYTES = 32768;
 constexpr uint32_t TM_O = 384;               // accumulator columns
@@ -59,7 +61,7 @@ struct __align__(16) Misc2 {
   uint64_t k_full[NKS], k_free[NKS], v_full[NVS], v_free[NVS];
   uint64_t s_full[2][NSB];                   // [owning warpgroup][buffer]: a waiter must see every phase of its barrier
   uint64_t p_a[2][NSB], p_b[2][NSB];         // [owning warpgroup = P V issuer][buffer]
-  uint64_t pv_issued[NSB];                   // leader only: P V of the tile in this buffer has been issued
+  uint64_t s_read[NSB];                      // leader only: S of the tile in this buffer is in registers (8 warps of the pair)
   uint64_t pv_turn[2];                       // leader only: issue token of the two P V issuers
   uint64_t o_full, acc_free, lse_ready;
   uint64_t t_full[2], t_free[2];
@@ -234,7 +236,7 @@ __device__ __forceinline__ void init_barriers2(Misc2& mi) {
   for (int s = 0; s < NKS; ++s) { mbar_init(&mi.k_full[s], 1); mbar_init(&mi.k_free[s], 1); }
   for (int s = 0; s < NVS; ++s) { mbar_init(&mi.v_full[s], 1); mbar_init(&mi.v_free[s], 1); }
   for (int s = 0; s < NSB; ++s) {
-    mbar_init(&mi.s_full[0][s], 1); mbar_init(&mi.s_full[1][s], 1); mbar_init(&mi.pv_issued[s], 1);
+    mbar_init(&mi.s_full[0][s], 1); mbar_init(&mi.s_full[1][s], 1); mbar_init(&mi.s_read[s], 8);
     for (int g = 0; g < 2; ++g) { mbar_init(&mi.p_a[g][s], 8); mbar_init(&mi.p_b[g][s], 8); }   // 4 warps of the owning warpgroup in each CTA
   }
   mbar_init(&mi.pv_turn[0], 1); mbar_init(&mi.pv_turn[1], 1);
@@ -384,10 +386,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const uint32_t q_u32 = smem_u32(cx.sQ[qb]);
           for (int j = 0; j < bk.n; ++j) {
             const int sb = cS % NSB;
-            // S overwrites the P of the tile that used this buffer three tiles ago.  The tensor pipe runs
-            // the MMAs in the order they were issued, so it is enough that P V of that tile has been
-            // ISSUED (ordered across the two issuing threads by the tcgen05 fences around the barrier).
-            WAIT2(&mi.pv_issued[sb], free_par(cS / NSB), W2_PVDONE);
+            // S(t) of a warpgroup overwrites its S(t-2): wait until that is in registers.  (P lives elsewhere.)
+            WAIT2(&mi.s_read[sb], free_par(cS / NSB), W2_PVDONE);
             const int s = cK % NKS;
             WAIT2(&mi.k_full[s], full_par(cK / NKS), W2_KFULL);
             tc_fence_after_sync();
@@ -467,21 +467,20 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int s = cS % NVS;                                            // one V stage per tile
             WAIT2(&mi.v_full[s], full_par(cS / NVS), W2_VFULL);
             const uint32_t v_u32 = rv_u32 + s * HALF_BYTES;
-            const uint32_t tP = cx.tmem + sb * TILE;
-            WAIT2(&mi.p_a[me][sb], full_par(cS / (2 * NSB)), W2_PA);           // keys 0..63 of P
+            const uint32_t tP = cx.tmem + TM_P + (cS & 1) * 64;
+            WAIT2(&mi.p_a[me][sb], full_par(cS / NSB), W2_PA);           // keys 0..63 of P
             WAIT2(&mi.pv_turn[me], me == 0 ? free_par(n_turn) : full_par(n_turn), W2_TURN);   // P V of tile cS-1 issued
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
               mma_ts_pair(cx.tmem + TM_O, tP + ks * 8, make_smem_desc_sw128(v_u32 + ks * 2048, 16384, 1024), idesc_pv,
                           j > 0 || ks > 0);
-            WAIT2(&mi.p_b[me][sb], full_par(cS / (2 * NSB)), W2_PB);           // keys 64..127
+            WAIT2(&mi.p_b[me][sb], full_par(cS / NSB), W2_PB);           // keys 64..127
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 4; ks < 8; ++ks)
               mma_ts_pair(cx.tmem + TM_O, tP + ks * 8, make_smem_desc_sw128(v_u32 + ks * 2048, 16384, 1024), idesc_pv, true);
             tc_fence_before_sync();
-            mbar_arrive(&mi.pv_issued[sb]);                                    // Q K^T may reuse this S/P buffer
             mbar_arrive(&mi.pv_turn[me ^ 1]);
             ++n_turn;
             mma_commit_pair(&mi.v_free[s]);
@@ -534,13 +533,16 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int owner = cS & 1;
           if (owner != hlf) continue;
           const int sb = cS % NSB;
-          WAIT2(&mi.s_full[owner][sb], full_par(cS / (2 * NSB)), W2_SFULL);   // its uses are 2 * NSB tiles apart
+          WAIT2(&mi.s_full[owner][sb], full_par(cS / NSB), W2_SFULL);
           tc_fence_after_sync();
           const uint32_t tS = cx.tmem + sb * TILE + lane_sel;
           uint32_t s[4][32];
 #pragma unroll
           for (int q = 0; q < 4; ++q) tmem_ld32(tS + q * 32, s[q]);
           tmem_wait_ld();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.s_read[sb], 0));   // Q K^T of this warpgroup's next tile may start
           const int vis = token - j * TILE + 1;                // visible columns (causal); >= 128: all
           if (vis < TILE) {
 #pragma unroll
@@ -595,6 +597,13 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               tmem_st8(tO + q * 8, o);
             }
           }
+          if (cS >= 2) {
+            // the P buffer of this warpgroup is free once P V of its previous tile has run; this wait also keeps
+            // the softmax at most one own tile ahead of the P V issuer, whose barriers have one phase bit
+            const uint32_t prev2 = cS - 2;
+            WAIT2(&mi.v_free[prev2 % NVS], full_par(prev2 / NVS), W2_PVDONE);
+            tc_fence_after_sync();
+          }
           const float neg_m = (m_new == -INFINITY) ? 0.0f : -m_new;
           const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), negm2 = pack_f32x2(neg_m, neg_m);
           uint64_t sum2[2] = {0ull, 0ull};
@@ -615,7 +624,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
               packed[i] = pack_bf16x2(p0, p1);
             }
-            tmem_st16(cx.tmem + sb * TILE + q * 16 + lane_sel, packed);   // P: 64 bf16 columns over S
+            tmem_st16(cx.tmem + TM_P + hlf * 64 + q * 16 + lane_sel, packed);   // P: 64 bf16 columns
             if (q == 1) {                                      // keys 0..63 are final: P V may start on them
               tmem_wait_st();
               tc_fence_before_sync();
