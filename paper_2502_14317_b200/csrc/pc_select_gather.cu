@@ -62,13 +62,14 @@ void launch_select_chunks(const float* score, int C, int m, int lower_is_better,
 //      order-preserving uint32 key and transposes its 32 x 32 bit matrix in registers: word b then
 //      holds bit b of all 32 keys (byte permutes for the 16- and 8-bit stages).
 //   2. The k-th largest key T is found bit by bit, most significant first.  On the bit slices a
-//      round is three instructions per thread (and, popc, redux) plus one shared-memory atomic
-//      per warp and one barrier, whatever the distribution of the scores; the masks of the keys
+//      round is three instructions per thread (and, popc, redux), one count per warp in shared memory,
+//      one barrier and one redux over the warps' counts, whatever the distribution of the scores (no
+//      atomics, no histogram hot spots); the masks of the keys
 //      > T and == T fall out.  The search stops as soon as every key still undecided belongs to
 //      the top k (with distinct scores after about log2(n_cand) rounds past their common prefix).
 //   3. One block scan over the per-chunk counts (eight counts packed in two words) gives every
-//      thread the output rank of its kept positions, which are stored straight to the index row in
-//      ascending order.  Only when the keys equal to T cannot all be kept does a second scan rank
+//      thread the output rank of its kept positions, which are put in ascending order in shared memory
+//      and written out coalesced (straight to the index row when k is too large to stage).  Only when the keys equal to T cannot all be kept does a second scan rank
 //      them first (ties go to the lower position).
 // HBM traffic: the row once (4 B per candidate) + 4 B per kept index.
 constexpr int SEL_KPT = 32;                                    // keys per thread
@@ -122,11 +123,6 @@ __device__ __forceinline__ int sel_ordered_offsets(uint32_t x, int lane, int war
   return total;
 }
 
-// One thread adds to a counter in shared memory (the compiler is not asked to aggregate over the warp again).
-__device__ __forceinline__ void sel_red_add(int* p, int v) {
-  asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(p))), "r"(v) : "memory");
-}
-
 // STAGE: the kept positions are first put in order in shared memory (k words) and written out coalesced;
 // otherwise (k too large for that) they are stored straight to the index row.
 template <bool CAL, bool STAGE>
@@ -135,7 +131,7 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
                                                                         int n_cand, int k, int* __restrict__ idx,
                                                                         const SelCalib cal) {
   extern __shared__ int sel_stage[];                           // STAGE: [min(k, n_cand)]
-  __shared__ int s_cnt[32];                                    // per bit: undecided keys of the row with that bit set
+  __shared__ int s_part[2][32];                                // [round parity][warp]: undecided keys of the warp with the bit set
   __shared__ int s_tot[2][32];
 
   const int row = blockIdx.x;                                  // r * Hkv + hkv
@@ -173,8 +169,6 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
       }
     }
   }
-  if (tid < 32) s_cnt[tid] = 0;
-  __syncthreads();                                             // the counters are cleared before the first round adds to them
 
   // Keys.  The order-preserving image of a score with bit pattern u is u ^ 0x80000000 for u >= 0 and ~u for
   // u < 0; the exclusive-or is applied to the bit slices inside the search (one operand more of a logic
@@ -245,18 +239,15 @@ __global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const fl
     const uint32_t slice = bit == 31 ? ~neg : key[31 - bit] ^ neg;   // this bit of the order-preserving images
     const uint32_t ones = active & slice;
     const int cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(ones));
-    if (lane == 0) sel_red_add(&s_cnt[bit], cnt);
+    int* const part = s_part[bit & 1];                         // per-warp counts, double-buffered over the rounds
+    if (lane == 0) part[warp] = cnt;
     __syncthreads();
-    const int tot = s_cnt[bit];                                // undecided keys with this bit set
-    if (tot >= need) {                                         // the k-th largest has this bit
-      active = ones;
-      n_active = tot;
-    } else {
-      above |= ones;
-      active &= ~slice;
-      need -= tot;
-      n_active -= tot;
-    }
+    const int tot = __reduce_add_sync(0xFFFFFFFFu, lane < nwarps ? part[lane] : 0);   // undecided keys with this bit set
+    const bool take = tot >= need;                             // the k-th largest has this bit
+    above |= take ? 0u : ones;
+    active = take ? ones : (active & ~slice);
+    need -= take ? 0 : tot;
+    n_active = take ? tot : n_active - tot;
   }
 
   // ---- 3. ordered emission
