@@ -78,6 +78,21 @@ def test_growing_logits_rescale_path(d):
     _run_and_compare(bits[0], bits[1], bits[2], w, 10000.0)
 
 
+@pytest.mark.parametrize("Hq,Hkv", [(4, 2), (2, 2), (6, 2)])
+def test_growing_logits_many_tiles(Hq, Hkv):
+    """The same stress over 13 key tiles, two chunks, even and odd group sizes: the softmax warpgroups, the three
+    issuing threads and the TMEM buffers go through many rounds in which a warpgroup stalls in the rescale path
+    while the other runs ahead, including across query blocks and the score sweep."""
+    rng = np.random.default_rng(7 + Hq)
+    C, L, w, d = 2, 1600, 64, 128
+    q = rng.standard_normal((C, L, Hq, d)).astype(np.float32)
+    k = rng.standard_normal((C, L, Hkv, d)).astype(np.float32)
+    v = rng.standard_normal((C, L, Hkv, d)).astype(np.float32)
+    k *= np.linspace(1.0, 60.0, L, dtype=np.float32)[None, :, None, None]
+    bits = [pc_inputs.f32_to_bf16_bits(x) for x in (q, k, v)]
+    _run_and_compare(bits[0], bits[1], bits[2], w, 10000.0)
+
+
 def test_deterministic_and_strided(cfg0_inputs):
     import paper_2502_14317_b200 as pc
     cfg, inp = cfg0_inputs
