@@ -75,6 +75,10 @@ void launch_select_chunks(const float* score, int C, int m, int lower_is_better,
 constexpr int SEL_KPT = 32;                                    // keys per thread
 constexpr int SEL_SPAN = 32 * SEL_KPT;                         // positions per warp
 constexpr int SEL_MAX_THREADS = 1024;                          // n_cand <= 32768
+#ifndef PC_SEL_SMALL_CTAS
+#define PC_SEL_SMALL_CTAS 5
+#endif
+constexpr int SEL_SMALL_CTAS = PC_SEL_SMALL_CTAS;
 
 // Attention calibration (Eq. 8): a candidate whose score exceeds the threshold of its region (first n_s
 // positions / last n_r positions / the rest) is evicted before the ranking.  +inf switches a region off.
@@ -125,8 +129,9 @@ __device__ __forceinline__ int sel_ordered_offsets(uint32_t x, int lane, int war
 
 // STAGE: the kept positions are first put in order in shared memory (k words) and written out coalesced;
 // otherwise (k too large for that) they are stored straight to the index row.
-template <bool CAL, bool STAGE>
-__global__ void __launch_bounds__(SEL_MAX_THREADS) select_tokens_kernel(const float* __restrict__ win_score,
+// SMALL: rows of at most 8192 candidates (256 threads), compiled for five CTAs per SM.
+template <bool CAL, bool STAGE, bool SMALL>
+__global__ void __launch_bounds__(SMALL ? 256 : SEL_MAX_THREADS, SMALL ? SEL_SMALL_CTAS : 1) select_tokens_kernel(const float* __restrict__ win_score,
                                                                         const int* __restrict__ kept, int Hkv, int L,
                                                                         int n_cand, int k, int* __restrict__ idx,
                                                                         const SelCalib cal) {
@@ -311,8 +316,15 @@ cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m,
   const size_t stage_bytes = sizeof(int) * (size_t)(k < n_cand ? k : n_cand);
   const bool stage = stage_bytes <= 40 * 1024;                 // within the default dynamic shared-memory limit
   const int grid = m * Hkv;
-#define PC_SELECT(C, S) \
-  select_tokens_kernel<C, S><<<grid, threads, S ? stage_bytes : 0, st>>>(win_score, kept, Hkv, L, n_cand, k, idx, cal)
+#define PC_SELECT(C, S)                                                                                               \
+  do {                                                                                                                \
+    if (threads <= 256)                                                                                               \
+      select_tokens_kernel<C, S, true><<<grid, threads, S ? stage_bytes : 0, st>>>(win_score, kept, Hkv, L, n_cand, k, \
+                                                                                    idx, cal);                        \
+    else                                                                                                              \
+      select_tokens_kernel<C, S, false><<<grid, threads, S ? stage_bytes : 0, st>>>(win_score, kept, Hkv, L, n_cand,   \
+                                                                                     k, idx, cal);                    \
+  } while (0)
   if (calib) {
     if (stage) PC_SELECT(true, true); else PC_SELECT(true, false);
   } else {
