@@ -316,7 +316,8 @@ def run_gpu(args, cfg):
                     "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
                     "d2h_bytes_per_step": int(h_out.numel()) * 2, "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": {"bound": "tensor", "kernel": "prefill_pair_kernel (+ RoPE table and key pre-pass inside the same call)",
+            "roofline": {"bound": "tensor", "kernel": ("prefill_pair_kernel" if (cfg.d == 128 and cfg.G % 2 == 0) else "prefill_attn_kernel") +
+                                   " (+ RoPE table and key pre-pass inside the same call)",
                          "achieved": ach_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                          "frac": ach_tflops / peaks["bf16_tflops_sustained"],
                          "frac_of_burst_peak": ach_tflops / peaks["bf16_tflops"],

@@ -157,8 +157,11 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
   prm.rope_tab32 = table32;
   prm.lse = lse; prm.win_lse = win_lse; prm.win_score = win_score;
   prm.status = status_word; prm.counter = counter;
-  // head size 128 runs on CTA pairs (cta_group::2); head size 64 on single CTAs with two blocks
-  const cudaError_t le = (d == 128 && dev.sm_count >= 2 && !PC_FORCE_SINGLE_CTA)
+  // head size 128 with an even number of q-heads per kv-head runs on CTA pairs (cta_group::2: the two CTAs take
+  // the same query tile of two heads that share K/V); head size 64 and odd group sizes (multi-head attention:
+  // one q-head per kv-head) run on single CTAs with two query blocks each
+  const bool even_group = ((desc->Hq / desc->Hkv) % 2) == 0;
+  const cudaError_t le = (d == 128 && even_group && dev.sm_count >= 2 && !PC_FORCE_SINGLE_CTA)
                              ? pc::launch_prefill_pair(maps, prm, dev.sm_count, st)
                              : pc::launch_prefill_attn(maps, prm, d, dev.sm_count, st);
   if (le != cudaSuccess) return PC_ERR_CUDA;

@@ -86,57 +86,43 @@ __device__ __forceinline__ uint32_t free_par(uint32_t n) { return (n & 1u) ^ 1u;
 // ------------------------------------------------------------------ work decomposition
 // Groups = (chunk, kv-head); the items of a group are ordered heaviest first; item 0 of a
 // group (the tail item) holds the query tiles with window rows for all G heads, then the sweep.
+// The two CTAs of a pair take the same query tile of two q-heads of the kv-head, so G must be even (an odd
+// group size would leave a pair with two different query tiles of one head, one of them walking a masked
+// key tile; such shapes run on the single-CTA kernel instead).
 struct Sched2 {
-  int T, t_w, ntt, G, P, even, ipg, n_lp, hp, n_pass;
+  int T, t_w, ntt, G, P, ipg, hp, n_pass;
 };
 __device__ __forceinline__ Sched2 make_sched2(const PrefillParams& p) {
   Sched2 s;
   s.T = (p.L + TILE - 1) / TILE;
   s.G = p.Hq / p.Hkv;
-  s.even = (s.G % 2 == 0);
   s.P = s.G / 2;
   s.t_w = (p.L - p.w) / TILE;
   s.ntt = s.T - s.t_w;
-  s.n_lp = 0;
-  if (s.even) {
-    s.ipg = 1 + s.t_w * s.P;
-  } else {
-    s.n_lp = s.T > 2 ? (s.T - 2 + 1) / 2 : 0;
-    s.ipg = 1 + s.n_lp * s.G;
-  }
-  const int cap = TILE / p.w, want = (s.G + 1) / 2;
+  s.ipg = 1 + s.t_w * s.P;
+  const int cap = TILE / p.w, want = s.G / 2;
   s.hp = cap < want ? cap : want;                         // window heads per CTA and sweep pass
   s.n_pass = (s.G + 2 * s.hp - 1) / (2 * s.hp);
   return s;
 }
 __device__ __forceinline__ int n_subitems2(const Sched2& s, int within) {
   if (within != 0) return 1;
-  return s.even ? s.P * s.ntt : s.G;
+  return s.P * s.ntt;
 }
 struct Blk {
   int h;       // q-head of this CTA's block
-  int t;       // query tile of this CTA's block; t >= T: no block (rows past the end, nothing stored)
+  int t;       // query tile of this CTA's block
   int n;       // key tiles the pair walks
 };
 __device__ __forceinline__ Blk decode_blk(const Sched2& s, int rank, int hkv, int within, int sub) {
   Blk b;
   const int h0 = hkv * s.G;
-  if (s.even) {
-    int pair, tile;
-    if (within == 0) { pair = sub / s.ntt; tile = s.T - 1 - (sub % s.ntt); }
-    else { const int x = within - 1; tile = s.t_w - 1 - x / s.P; pair = x % s.P; }
-    b.h = h0 + 2 * pair + rank;
-    b.t = tile;
-    b.n = tile + 1;
-  } else {
-    int g, ta, tb;
-    if (within == 0) { g = sub; if (s.T >= 2) { ta = s.T - 2; tb = s.T - 1; } else { ta = 0; tb = s.T; } }
-    else { const int x = within - 1; g = x % s.G; const int thi = s.T - 3 - 2 * (x / s.G); ta = thi - 1; tb = thi; }
-    b.h = h0 + g;
-    b.n = (tb < s.T ? tb : ta) + 1;
-    if (ta < 0) ta = s.T;
-    b.t = rank ? tb : ta;
-  }
+  int pair, tile;
+  if (within == 0) { pair = sub / s.ntt; tile = s.T - 1 - (sub % s.ntt); }
+  else { const int x = within - 1; tile = s.t_w - 1 - x / s.P; pair = x % s.P; }
+  b.h = h0 + 2 * pair + rank;
+  b.t = tile;
+  b.n = tile + 1;
   return b;
 }
 
@@ -817,6 +803,7 @@ cudaError_t launch_prefill_pair(const CUtensorMap* maps, const PrefillParams& pr
   }
   const int grid = (sm_count / 2) * 2;
   if (grid < 2) return cudaErrorInvalidConfiguration;
+  if ((prm.Hq / prm.Hkv) % 2 != 0) return cudaErrorInvalidValue;   // the pair kernel takes even group sizes
   prefill_pair_kernel<<<grid, NT2, SMEM2_BYTES, st>>>(maps[0], maps[5], maps[1], maps[2], maps[3], maps[4], prm);
   return cudaGetLastError();
 }
