@@ -27,9 +27,6 @@
 #include "pc_attn.h"
 #include "pc_sm100.cuh"
 
-#ifndef PC_POLY_PAIRS_PER_8
-#define PC_POLY_PAIRS_PER_8 2
-#endif
 
 namespace pc {
 
@@ -42,7 +39,6 @@ constexpr int WARP_MMA = 9;                 // issuer of block 0; WARP_MMA + 1 i
 constexpr int NS = 4;                       // K/V ring stages
 constexpr float LAZY_RESCALE = 8.0f;        // log2 units
 constexpr int ITEM_DONE = -1;
-constexpr int POLY_PAIRS_PER_8 = PC_POLY_PAIRS_PER_8;   // of every 8 logit pairs, how many take the polynomial exp2
 
 // where-codes stored in the status word when a wait gives up
 enum { W_ITEM = 101, W_QFULL, W_QROT, W_QFREE, W_KVFULL, W_KVFREE, W_SFULL, W_PFULL, W_OFULL, W_ACCFREE, W_TFULL, W_TFREE, W_TURN, W_PHALF };
@@ -215,12 +211,8 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_taddr, uint32_t o_taddr,
       const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[q][2 * j]), __uint_as_float(s[q][2 * j + 1])), scale2, negm2);
       float x0, x1, p0, p1;
       unpack_f32x2(x2, x0, x1);
-      if (((j * POLY_PAIRS_PER_8) % 8) < POLY_PAIRS_PER_8) {
-        exp2_poly_x2(x0, x1, p0, p1);                             // FMA pipe
-      } else {
-        p0 = fast_exp2(x0);                                       // MUFU pipe
-        p1 = fast_exp2(x1);
-      }
+      p0 = fast_exp2(x0);                                         // MUFU pipe
+      p1 = fast_exp2(x1);
       sum2[j & 1] = add_f32x2(sum2[j & 1], pack_f32x2(p0, p1));
       packed[j] = pack_bf16x2(p0, p1);
     }

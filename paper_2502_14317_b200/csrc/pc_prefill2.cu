@@ -32,9 +32,6 @@
 #ifndef PC2_EARLY_ROT
 #define PC2_EARLY_ROT 1
 #endif
-#ifndef PC2_POLY_PAIRS_PER_8
-#define PC2_POLY_PAIRS_PER_8 0
-#endif
 
 namespace pc {
 
@@ -51,7 +48,6 @@ constexpr int HALF_BYTES = 16384;            // 64 keys x 128 d of K, or 128 key
 constexpr int Q_BYTES = 32768;
 constexpr uint32_t TM_O = 384;               // accumulator columns
 constexpr float LAZY_RESCALE = 8.0f;         // log2 units
-constexpr int POLY_PAIRS_PER_8 = PC2_POLY_PAIRS_PER_8;
 
 enum { W2_QFULL = 201, W2_QREADY, W2_QFREE, W2_KFULL, W2_KFREE, W2_VFULL, W2_VFREE, W2_SFULL, W2_PA, W2_PB,
        W2_PVDONE, W2_OFULL, W2_ACCFREE, W2_LSE, W2_TFULL, W2_TFREE, W2_MPUB, W2_TURN };
@@ -601,12 +597,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[q][2 * i]), __uint_as_float(s[q][2 * i + 1])), scale2, negm2);
               float x0, x1, p0, p1;
               unpack_f32x2(x2, x0, x1);
-              if (((i * POLY_PAIRS_PER_8) % 8) < POLY_PAIRS_PER_8) {
-                exp2_poly_x2(x0, x1, p0, p1);
-              } else {
-                p0 = fast_exp2(x0);
-                p1 = fast_exp2(x1);
-              }
+              p0 = fast_exp2(x0);                                // MUFU pipe
+              p1 = fast_exp2(x1);
               sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
               packed[i] = pack_bf16x2(p0, p1);
             }

@@ -292,29 +292,6 @@ __device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
   return d;
 }
 
-// 2^x for a pair of values on the FMA pipe (no MUFU): round x to the nearest integer n with the
-// 1.5 * 2^23 trick, evaluate a cubic for 2^f on f = x - n in [-0.5, 0.5] (minimax in relative
-// error, 8e-5) and add n to the exponent field.  x is clamped at -126 (result ~ 0); x must be < 128.
-__device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& y0, float& y1) {
-  const float MAGIC = 12582912.0f;
-  const uint64_t magic2 = pack_f32x2(MAGIC, MAGIC), nmagic2 = pack_f32x2(-MAGIC, -MAGIC);
-  const uint64_t neg1 = pack_f32x2(-1.0f, -1.0f);
-  const uint64_t c0 = pack_f32x2(0.99992806f, 0.99992806f), c1 = pack_f32x2(0.69326097f, 0.69326097f);
-  const uint64_t c2 = pack_f32x2(0.24261114f, 0.24261114f), c3 = pack_f32x2(0.055171665f, 0.055171665f);
-  const uint64_t x2 = pack_f32x2(fmaxf(x0, -126.0f), fmaxf(x1, -126.0f));
-  const uint64_t t2 = add_f32x2(x2, magic2);                 // low mantissa bits hold n
-  const uint64_t n2 = add_f32x2(t2, nmagic2);
-  const uint64_t f2 = fma_f32x2(n2, neg1, x2);
-  uint64_t p2 = fma_f32x2(c3, f2, c2);
-  p2 = fma_f32x2(p2, f2, c1);
-  p2 = fma_f32x2(p2, f2, c0);
-  float p0, p1, t0, t1;
-  unpack_f32x2(p2, p0, p1);
-  unpack_f32x2(t2, t0, t1);
-  y0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-  y1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
-}
-
 // Round an fp64 value to bf16, ties to even, in one rounding (no fp32 detour).
 __device__ __forceinline__ uint16_t f64_to_bf16_rne(double x) {
   // fp64 -> fp32 with round-to-odd keeps enough information for a second, exact RNE step
