@@ -299,8 +299,8 @@ def run_gpu(args, cfg):
         # profiles/prefill_pair_kernel_cfg1_C2_ncu_full.md (2 of 16 chunks captured, scaled by the chunk count)
         traffic, traffic_note = args.traffic_bytes, "command line"
         if traffic is None and args.workload == "cfg1":
-            traffic = 350.35e6 / 2 * cfg.C
-            traffic_note = "ncu dram__bytes_read+write of a 2-chunk launch (350.35 MB) scaled to %d chunks" % cfg.C
+            traffic = 354.24e6 / 2 * cfg.C
+            traffic_note = "ncu dram__bytes_read+write of a 2-chunk launch (354.24 MB) scaled to %d chunks" % cfg.C
         flops = prefill_flops(cfg)
         ach_tflops = flops / (stage_ms["prefill_attn"] * 1e-3) / 1e12
         gather_bytes = 2.0 * (2 * cfg.Hkv * cfg.m * cfg.k * cfg.d * 2)
