@@ -17,6 +17,7 @@ import argparse
 import dataclasses
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -43,6 +44,40 @@ def load_peaks():
         return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
                 "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def choose_bf16_peak(peaks: dict, clocks: dict | None, timed_region_s: float) -> tuple[float, str]:
+    """The bf16 roofline denominator that fits this run: the burst cuBLAS figure unless the run's own clock
+    record shows the power-managed regime of the sustained figure (a timed region of a second or more whose
+    median SM clock sits more than 5 % below the maximum)."""
+    sm, mx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    power_managed = bool(sm and mx and sm < 0.95 * mx)
+    if timed_region_s >= 1.0 and power_managed:
+        return peaks["bf16_tflops_sustained"], (f"{peaks['source']} cuBLAS bf16, sustained: timed region {timed_region_s:.2f} s at a "
+                                                f"median SM clock of {sm:.0f} of {mx:.0f} MHz")
+    why = f"timed region {timed_region_s:.2f} s" + (f", median SM clock {sm:.0f} of {mx:.0f} MHz" if sm and mx else ", no clock samples")
+    return peaks["bf16_tflops"], f"{peaks['source']} cuBLAS bf16, burst: {why}"
+
+
+def recorded_traffic(kernel_sources: list[str], profile: str, scale: float):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary `profile` (a line
+    `dram_bytes_captured: N` and a line `kernel_source_sha256: H` over the listed source files).  Returns
+    (bytes scaled to this launch, note), or (None, why) when the kernel sources changed since the capture."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", profile)
+    try:
+        text = open(path).read()
+        captured = float(re.search(r"dram_bytes_captured:\s*([0-9.eE+]+)", text).group(1))
+        want = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text).group(1)
+    except Exception:
+        return None, f"no machine-readable traffic record in profiles/{profile}"
+    h = hashlib.sha256()
+    for f in kernel_sources:
+        with open(os.path.join(ROOT, "paper_2502_14317_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    if h.hexdigest() != want:
+        return None, f"kernel sources changed since the capture in profiles/{profile}"
+    return captured * scale, f"ncu dram__bytes_read+write of the capture in profiles/{profile} ({captured / 1e6:.2f} MB) x {scale:g}"
 
 
 def prefill_flops(cfg) -> float:
@@ -175,6 +210,34 @@ def replica_throughput(units_per_rank: float, world: int, max_ms_per_step: float
     return world * units_per_rank / (max_ms_per_step * 1e-3)
 
 
+def worker_environments(n: int, port: int, base_env=None) -> list:
+    """Environments of the n replica processes of one node (one process per GPU, rendezvous on 127.0.0.1)."""
+    envs = []
+    for r in range(n):
+        e = dict(os.environ if base_env is None else base_env)
+        e.update({"RANK": str(r), "LOCAL_RANK": str(r), "WORLD_SIZE": str(n), "LOCAL_WORLD_SIZE": str(n),
+                  "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+        envs.append(e)
+    return envs
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_workers(cmd: list, n: int, port=None) -> int:
+    """Start `cmd` n times as ranks 0..n-1 (rank 0 inherits stdout, the others' stdout is dropped: rank 0 prints the
+    line), wait for all of them, return the largest exit code."""
+    port = free_port() if port is None else port
+    procs = []
+    for r, env in enumerate(worker_environments(n, port)):
+        procs.append(subprocess.Popen(cmd, env=env, stdout=None if r == 0 else subprocess.DEVNULL))
+    return max(abs(p.wait()) for p in procs)
+
+
 # --------------------------------------------------------------------------------------- GPU leg
 def run_gpu(args, cfg):
     import torch
@@ -295,14 +358,21 @@ def run_gpu(args, cfg):
     value = replica_throughput(tokens, world, ms_per_step)
 
     if rank == 0:
-        # DRAM bytes per launch of the dominant kernel, from the ncu capture summarised in
-        # profiles/prefill_pair_kernel_cfg1_C2_ncu_full.md (2 of 16 chunks captured, scaled by the chunk count)
+        # DRAM bytes per launch of the dominant kernel: read from the committed ncu summary (a 2-chunk launch
+        # of the same shape, scaled by the chunk count); null once the kernel sources differ from the captured ones
+        pair_path = cfg.d == 128 and cfg.G % 2 == 0
         traffic, traffic_note = args.traffic_bytes, "command line"
-        if traffic is None and args.workload == "cfg1":
-            traffic = 354.24e6 / 2 * cfg.C
-            traffic_note = "ncu dram__bytes_read+write of a 2-chunk launch (354.24 MB) scaled to %d chunks" % cfg.C
+        if traffic is None:
+            if pair_path and cfg.L == 8192 and cfg.Hq == 32 and cfg.Hkv == 8:
+                traffic, traffic_note = recorded_traffic(["pc_prefill2.cu", "pc_sm100.cuh"],
+                                                         "prefill_pair_kernel_cfg1_C2_ncu_full.md", cfg.C / 2.0)
+            else:
+                traffic_note = "no ncu capture of this shape"
         flops = prefill_flops(cfg)
         ach_tflops = flops / (stage_ms["prefill_attn"] * 1e-3) / 1e12
+        peak_tflops, peak_note = choose_bf16_peak(peaks, clocks, total_ms * 1e-3)
+        sm_count = props.multi_processor_count
+        sm_mhz = (clocks or {}).get("sm_mhz")
         gather_bytes = 2.0 * (2 * cfg.Hkv * cfg.m * cfg.k * cfg.d * 2)
         sel_bytes = 4.0 * cfg.m * cfg.Hkv * (cfg.ctx + cfg.k)
         par_flops = 4.0 * cfg.d * (cfg.m * cfg.k + (w + 1) / 2) * w * cfg.Hq
@@ -316,13 +386,15 @@ def run_gpu(args, cfg):
                     "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
                     "d2h_bytes_per_step": int(h_out.numel()) * 2, "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": {"bound": "tensor", "kernel": ("prefill_pair_kernel" if (cfg.d == 128 and cfg.G % 2 == 0) else "prefill_attn_kernel") +
+            "roofline": {"bound": "tensor", "kernel": ("prefill_pair_kernel" if pair_path else "prefill_attn_kernel") +
                                    " (+ RoPE table and key pre-pass inside the same call)",
-                         "achieved": ach_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                         "frac": ach_tflops / peaks["bf16_tflops_sustained"],
+                         "achieved": ach_tflops, "peak": peak_tflops, "unit": "TFLOP/s",
+                         "frac": ach_tflops / peak_tflops,
                          "frac_of_burst_peak": ach_tflops / peaks["bf16_tflops"],
+                         "frac_of_sustained_peak": ach_tflops / peaks["bf16_tflops_sustained"],
                          "frac_of_nominal_2250": ach_tflops / 2250.0,
-                         "peak_source": peaks["source"] + " cuBLAS bf16, sustained (kernel timed inside a long step)",
+                         "peak_source": peak_note,
+                         "flop_per_clk_per_sm": (ach_tflops * 1e12 / (sm_mhz * 1e6 * sm_count)) if sm_mhz else None,
                          "algorithmic_flops_per_launch": flops, "ms_per_launch": stage_ms["prefill_attn"],
                          "traffic": traffic, "traffic_note": traffic_note},
             "stages": {
@@ -501,6 +573,9 @@ def main():
         print(json.dumps({"extra": extra_measurements(pc, torch, dev, load_peaks(), only=args.extra_only,
                                                       select_chunks=args.select_chunks)}))
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started without a launcher: become the launcher of --gpus replicas, one process per GPU
+        sys.exit(spawn_workers([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus))
     if args.impl == "reference":
         # the oracle takes ~20 s per sample: bound the run to a few minutes whatever K and W say
         args.steps_ref = max(1, min(args.steps, 3))

@@ -94,6 +94,22 @@ PC_API int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q,
                               int32_t* status_word, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------
+ * RoPE with position reuse on its own.  Paper: Sec. 3.1 "Parallel attention" (the position
+ * encodings of every chunk restart at 0).
+ *     y[c, p, h, :] = bf16( RoPE(x[c, p, h, :]) at position p ),  pairs (t, t + d/2),
+ *     angle p * theta^(-2t/d), evaluated so that the result equals the fp64 rotation
+ *     rounded once to bf16.
+ * This is the rotation pc_chunk_prefill_attn applies to queries in its tile prologue and to
+ * keys in its pre-pass (for d = 128 it runs the very routine of the tile prologue), offered
+ * for callers that want rotated queries or keys as tensors.  x, y [C,L,H,d] bf16 contiguous.
+ * Workspace: pc_rope_position_reuse_workspace_bytes(L, d) (cos/sin tables).
+ */
+PC_API size_t pc_rope_position_reuse_workspace_bytes(int32_t L, int32_t d);
+
+PC_API int32_t pc_rope_position_reuse(const void* x, int32_t C, int32_t L, int32_t H, int32_t d, float rope_theta,
+                                void* y, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------
  * Stand-in for the chunk self-information I_c of Eq. 3 in a single-layer setting
  * (the true I_c = -log P(X^q | X^c) needs the whole model; it enters pc_select_chunks
  * as an input array).  chunk_score[c] = - mean over q-heads and window rows of

@@ -48,6 +48,10 @@ def load_library():
     lib.pc_chunk_prefill_attn_workspace_bytes.argtypes = [POINTER(_PrefillDesc), c_int32]
     lib.pc_chunk_prefill_attn.restype = c_int32
     lib.pc_chunk_prefill_attn.argtypes = [POINTER(_PrefillDesc)] + [c_void_p] * 10 + [c_size_t, c_void_p]
+    lib.pc_rope_position_reuse_workspace_bytes.restype = c_size_t
+    lib.pc_rope_position_reuse_workspace_bytes.argtypes = [c_int32, c_int32]
+    lib.pc_rope_position_reuse.restype = c_int32
+    lib.pc_rope_position_reuse.argtypes = [c_void_p] + [c_int32] * 4 + [c_float, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.pc_chunk_score_from_lse.restype = c_int32
     lib.pc_chunk_score_from_lse.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
     lib.pc_select_chunks.restype = c_int32
@@ -148,18 +152,30 @@ def chunk_prefill_attn(q, k, v, *, w, rope_theta, softmax_scale=0.0, want_lse=Fa
         status = torch.zeros(1, dtype=torch.int32, device=dev)
     desc = _make_desc(q, k, v, o, w, rope_theta, softmax_scale)
     need = int(lib.pc_chunk_prefill_attn_workspace_bytes(ctypes.byref(desc), 0))
-    if need == 0:
-        _check(lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(k_rot), _ptr(lse),
-                                         _ptr(win_score), _ptr(win_lse), _ptr(status), None, 0, _stream()),
-               "pc_chunk_prefill_attn")
-    if workspace is None or workspace.numel() < need:
-        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    if workspace is None or workspace.numel() < need:          # need == 0: a bad descriptor, which the call below names
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
     rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(k_rot), _ptr(lse),
                                    _ptr(win_score), _ptr(win_lse), _ptr(status), _ptr(workspace), workspace.numel(),
                                    _stream())
     _check(rc, "pc_chunk_prefill_attn")
     return {"o": o, "k_rot": k_rot, "win_score": win_score, "win_lse": win_lse, "lse": lse, "status": status,
             "workspace": workspace}
+
+
+def rope_position_reuse(x, *, rope_theta, out=None, workspace=None):
+    """pc_rope_position_reuse: x [C,L,H,d] bf16 contiguous -> the rotated tensor (positions 0..L-1 in every chunk)."""
+    lib = load_library()
+    _need_cuda(x)
+    if not x.is_contiguous():
+        raise PcError("pc_rope_position_reuse takes a contiguous tensor")
+    C, L, H, d = x.shape
+    out = torch.empty_like(x) if out is None else out
+    need = int(lib.pc_rope_position_reuse_workspace_bytes(L, d))
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=x.device)
+    _check(lib.pc_rope_position_reuse(_ptr(x), C, L, H, d, float(rope_theta), _ptr(out), _ptr(workspace), workspace.numel(),
+                                      _stream()), "pc_rope_position_reuse")
+    return out
 
 
 def chunk_score_from_lse(win_lse, out=None):

@@ -54,7 +54,7 @@ PrefillLayout prefill_layout(const pc_prefill_desc* d, bool krot_in_ws) {
   size_t off = 0;
   l.off_counter = off; off += ALIGN;
   l.off_table = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(double2));
-  l.off_table32 = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(float2));
+  l.off_table32 = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(float4));
   l.off_krot = off;
   if (krot_in_ws) off += align_up((size_t)d->C * d->L * d->Hkv * d->d * 2);
   l.total = off;
@@ -122,7 +122,7 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   int* counter = reinterpret_cast<int*>(ws + lay.off_counter);
   double2* table = reinterpret_cast<double2*>(ws + lay.off_table);
-  float2* table32 = reinterpret_cast<float2*>(ws + lay.off_table32);
+  float4* table32 = reinterpret_cast<float4*>(ws + lay.off_table32);
   void* krot = krot_in_ws ? static_cast<void*>(ws + lay.off_krot) : k_rot;
 
   // tensor maps (innermost first: d, head, token, chunk)
@@ -154,7 +154,7 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
   const double scale = desc->softmax_scale > 0.0f ? (double)desc->softmax_scale : 1.0 / std::sqrt((double)d);
   prm.scale_log2 = (float)(scale * 1.4426950408889634);
   prm.rope_tab = table;
-  prm.rope_tab32 = table32;
+  prm.rope_tab4 = table32;
   prm.lse = lse; prm.win_lse = win_lse; prm.win_score = win_score;
   prm.status = status_word; prm.counter = counter;
   // head size 128 with an even number of q-heads per kv-head runs on CTA pairs (cta_group::2: the two CTAs take
@@ -165,6 +165,34 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
                              ? pc::launch_prefill_pair(maps, prm, dev.sm_count, st)
                              : pc::launch_prefill_attn(maps, prm, d, dev.sm_count, st);
   if (le != cudaSuccess) return PC_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------ RoPE with position reuse
+size_t pc_rope_position_reuse_workspace_bytes(int32_t L, int32_t d) {
+  if (L < 1 || (d != 64 && d != 128)) return 0;
+  return align_up((size_t)L * (d / 2) * sizeof(double2)) + align_up((size_t)L * (d / 2) * sizeof(float4));
+}
+
+int32_t pc_rope_position_reuse(const void* x, int32_t C, int32_t L, int32_t H, int32_t d, float rope_theta, void* y,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+  if (!x || !y || C < 1 || L < 1 || H < 1 || !(rope_theta > 0.0f)) return PC_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(y) || !aligned16(workspace)) return PC_ERR_INVALID_ARG;
+  if ((int64_t)C * H > (1 << 24) || L > (1 << 24)) return PC_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < pc_rope_position_reuse_workspace_bytes(L, d)) return PC_ERR_WORKSPACE;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  double2* table = reinterpret_cast<double2*>(ws);
+  float4* table4 = reinterpret_cast<float4*>(ws + align_up((size_t)L * (d / 2) * sizeof(double2)));
+  pc::launch_rope_table(table, table4, L, d, (double)rope_theta, 0, st);
+  if (d == 128) {
+    pc::launch_rope_tiles(x, y, table4, table, C, L, H, st);
+  } else {
+    const long long str[3] = {(long long)L * H * d, (long long)H * d, d};
+    pc::launch_rope_keys(x, str, y, table, C, L, H, d, st);
+  }
   return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
 }
 

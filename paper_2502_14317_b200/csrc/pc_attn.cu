@@ -943,13 +943,10 @@ __global__ void __launch_bounds__(256) parallel_merge_kernel(const float* __rest
 // ====================================================================================
 template <int D>
 static cudaError_t launch_prefill_t(const CUtensorMap* maps, const PrefillParams& prm, int grid, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         Cfg<D>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  // the opt-in to large dynamic shared memory is a per-device attribute of the function: set it on every call
+  // (a host-side call of a few hundred nanoseconds) rather than remember which devices have it
+  if (cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Cfg<D>::SMEM_BYTES); e != cudaSuccess) return e;
   prefill_attn_kernel<D><<<grid, NUM_THREADS, Cfg<D>::SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
   return cudaGetLastError();
 }
@@ -960,13 +957,10 @@ cudaError_t launch_prefill_attn(const CUtensorMap* maps, const PrefillParams& pr
 
 template <int D>
 static cudaError_t launch_parallel_t(const CUtensorMap* maps, const ParallelParams& prm, int grid, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(parallel_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         Cfg<D>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  // the opt-in to large dynamic shared memory is a per-device attribute of the function: set it on every call
+  // (a host-side call of a few hundred nanoseconds) rather than remember which devices have it
+  if (cudaError_t e = cudaFuncSetAttribute(parallel_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Cfg<D>::SMEM_BYTES); e != cudaSuccess) return e;
   parallel_attn_kernel<D><<<grid, NUM_THREADS, Cfg<D>::SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -11,7 +11,7 @@ struct PrefillParams {
   int C, L, w, Hq, Hkv;
   float scale_log2;              // softmax scale * log2(e)
   const double2* rope_tab;       // [L][d/2] (cos, sin)
-  const float2* rope_tab32;      // the same table rounded to fp32
+  const float4* rope_tab4;       // the same entries as (cos_hi, sin_hi, cos_lo, sin_lo): fp32 head + tail
   float* lse;                    // [C,Hq,L] or null
   float* win_lse;                // [C,Hq,w]
   float* win_score;              // [C,Hkv,L]

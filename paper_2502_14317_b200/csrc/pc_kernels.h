@@ -7,12 +7,16 @@
 namespace pc {
 
 // ---- pc_rope.cu
-// cos/sin table: tab[p * (d/2) + t] = (cos, sin)(  (pos0 + p) * theta^(-2t/d) ), fp64; tab32 (may be null): the
-// same entries rounded to fp32.
-void launch_rope_table(double2* tab, float2* tab32, int n_pos, int d, double theta, int pos0, cudaStream_t st);
+// cos/sin table: tab[p * (d/2) + t] = (cos, sin)(  (pos0 + p) * theta^(-2t/d) ), fp64; tab4 (may be null): the
+// same entries as (cos_hi, sin_hi, cos_lo, sin_lo), fp32 head + fp32 tail of each value.
+void launch_rope_table(double2* tab, float4* tab4, int n_pos, int d, double theta, int pos0, cudaStream_t st);
 // k_rot[c,p,h,:] = bf16( RoPE(k[c,p,h,:], position p) ), rotation evaluated in fp64.
 void launch_rope_keys(const void* k, const long long k_stride[3], void* k_rot, const double2* tab, int C, int L,
                       int Hkv, int d, cudaStream_t st);
+
+// y[c,p,h,:] = bf16( RoPE(x[c,p,h,:], position p) ) for head size 128, tile by tile with the routine of the
+// attention kernel's query prologue (fp32 with exact fallbacks: same bits as the fp64 rotation).
+void launch_rope_tiles(const void* x, void* y, const float4* tab4, const double2* tab, int C, int L, int H, cudaStream_t st);
 
 // ---- pc_select_gather.cu
 void launch_chunk_score(const float* win_lse, int C, int n_per_chunk, float* score, cudaStream_t st);

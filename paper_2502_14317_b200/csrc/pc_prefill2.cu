@@ -28,10 +28,7 @@
 #include "pc_kernels.h"
 #include "pc_attn.h"
 #include "pc_sm100.cuh"
-
-#ifndef PC2_EARLY_ROT
-#define PC2_EARLY_ROT 1
-#endif
+#include "pc_rope_tile.cuh"
 
 namespace pc {
 
@@ -85,8 +82,28 @@ __device__ __forceinline__ uint32_t free_par(uint32_t n) { return (n & 1u) ^ 1u;
 // The two CTAs of a pair take the same query tile of two q-heads of the kv-head, so G must be even (an odd
 // group size would leave a pair with two different query tiles of one head, one of them walking a masked
 // key tile; such shapes run on the single-CTA kernel instead).
+// Division of n < 2^31 by a fixed divisor as a multiplication (round-up method with a 32-bit multiplier).
+struct FastDiv {
+  uint32_t d, mul, shr;
+  __device__ __forceinline__ void init(uint32_t div) {
+    d = div;
+    uint32_t l = 0;
+    while ((1u << l) < div) ++l;                           // ceil(log2(div))
+    shr = 31u + l;
+    mul = static_cast<uint32_t>(((1ull << shr) + div - 1) / div);
+  }
+  __device__ __forceinline__ int quot(int n) const {
+    return static_cast<int>((static_cast<uint64_t>(static_cast<uint32_t>(n)) * mul) >> shr);
+  }
+  __device__ __forceinline__ void divmod(int n, int& q, int& r) const {
+    q = quot(n);
+    r = n - q * static_cast<int>(d);
+  }
+};
+
 struct Sched2 {
   int T, t_w, ntt, G, P, ipg, hp, n_pass;
+  FastDiv d_ipg, d_hkv, d_ntt, d_P;
 };
 __device__ __forceinline__ Sched2 make_sched2(const PrefillParams& p) {
   Sched2 s;
@@ -99,6 +116,7 @@ __device__ __forceinline__ Sched2 make_sched2(const PrefillParams& p) {
   const int cap = TILE / p.w, want = s.G / 2;
   s.hp = cap < want ? cap : want;                         // window heads per CTA and sweep pass
   s.n_pass = (s.G + 2 * s.hp - 1) / (2 * s.hp);
+  s.d_ipg.init(s.ipg); s.d_hkv.init(p.Hkv); s.d_ntt.init(s.ntt); s.d_P.init(s.P);
   return s;
 }
 __device__ __forceinline__ int n_subitems2(const Sched2& s, int within) {
@@ -114,8 +132,8 @@ __device__ __forceinline__ Blk decode_blk(const Sched2& s, int rank, int hkv, in
   Blk b;
   const int h0 = hkv * s.G;
   int pair, tile;
-  if (within == 0) { pair = sub / s.ntt; tile = s.T - 1 - (sub % s.ntt); }
-  else { const int x = within - 1; tile = s.t_w - 1 - x / s.P; pair = x % s.P; }
+  if (within == 0) { int rem; s.d_ntt.divmod(sub, pair, rem); tile = s.T - 1 - rem; }
+  else { int q; s.d_P.divmod(within - 1, q, pair); tile = s.t_w - 1 - q; }
   b.h = h0 + 2 * pair + rank;
   b.t = tile;
   b.n = tile + 1;
@@ -150,63 +168,6 @@ __device__ __forceinline__ void mbar_wait_cluster(uint64_t* bar, uint32_t parity
         return;
       }
     }
-  }
-}
-
-// RoPE of 16 rows of a 128-byte-swizzled [128 x 128] bf16 Q tile (two atoms of 64 columns) by one warp:
-// rows row0 .. row0 + 15, row i at position pos_of(i) (negative: leave the row alone).  Lane l takes the
-// pairs (t, t + 64) for t = 2l, 2l + 1 of a row, so a warp reads a row of the cos/sin table as one
-// contiguous block (with a thread per row every lane reads its own table row: 32 cache lines per load
-// instruction), and the table reads of all 16 rows are in flight together.
-// The result is the fp64 rotation rounded once to bf16, bit for bit, but fp64 arithmetic (and the
-// fp32 <-> fp64 conversions around it, which run at a fraction of the fp32 rate) is only used where it
-// matters: the rotation is first evaluated in fp32 with the fp32 copy of the table; its error is below
-// 2^-22 (|x1| + |x2|), so when y - tol and y + tol with tol = 2^-21 (|x1| + |x2|) round to the same bf16
-// value, that value is the correctly rounded one.  Otherwise (about one output in a few thousand) the
-// pair is redone in fp64.
-template <typename PosOf>
-__device__ __forceinline__ void rope_rows_warp(uint8_t* tile, int row0, int lane, const double2* __restrict__ tab,
-                                               const float2* __restrict__ tab32, PosOf pos_of) {
-  // all reads first, then the arithmetic, then all writes: reads and writes of the tile go through
-  // pointers the compiler cannot tell apart, so a write in the middle would serialise the rows
-  float4 cs[16];
-  uint32_t lo[16], hi[16];
-  int pos[16];
-  uint8_t* const lo_base = tile + (lane & 3) * 4;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    pos[i] = pos_of(row0 + i);
-    cs[i] = __ldg(reinterpret_cast<const float4*>(tab32 + (size_t)(pos[i] < 0 ? 0 : pos[i]) * (D / 2) + 2 * lane));
-    const uint8_t* lo_p = lo_base + sw128_offset(row0 + i, lane >> 2);
-    lo[i] = *reinterpret_cast<const uint32_t*>(lo_p);
-    hi[i] = *reinterpret_cast<const uint32_t*>(lo_p + 16384);
-  }
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const float a0 = __uint_as_float(lo[i] << 16), a1 = __uint_as_float(lo[i] & 0xFFFF0000u);   // x1 of pairs 2l, 2l + 1
-    const float b0 = __uint_as_float(hi[i] << 16), b1 = __uint_as_float(hi[i] & 0xFFFF0000u);   // x2
-    const float c0 = cs[i].x, s0 = cs[i].y, c1 = cs[i].z, s1 = cs[i].w;
-    const float yl0 = fmaf(-b0, s0, a0 * c0), yh0 = fmaf(a0, s0, b0 * c0);
-    const float yl1 = fmaf(-b1, s1, a1 * c1), yh1 = fmaf(a1, s1, b1 * c1);
-    const float tol0 = 4.76837158203125e-7f * (fabsf(a0) + fabsf(b0)), tol1 = 4.76837158203125e-7f * (fabsf(a1) + fabsf(b1));
-    uint32_t rl = pack_bf16x2(yl0 - tol0, yl1 - tol1), rh = pack_bf16x2(yh0 - tol0, yh1 - tol1);
-    const uint32_t rl_up = pack_bf16x2(yl0 + tol0, yl1 + tol1), rh_up = pack_bf16x2(yh0 + tol0, yh1 + tol1);
-    if ((rl != rl_up || rh != rh_up) && pos[i] >= 0) {         // too close to a rounding boundary: exact
-      const double2* tab_row = tab + (size_t)pos[i] * (D / 2) + 2 * lane;
-      const double2 t0 = __ldg(tab_row), t1 = __ldg(tab_row + 1);
-      const double da0 = (double)a0, da1 = (double)a1, db0 = (double)b0, db1 = (double)b1;
-      rl = (uint32_t)f64_to_bf16_rne(da0 * t0.x - db0 * t0.y) | ((uint32_t)f64_to_bf16_rne(da1 * t1.x - db1 * t1.y) << 16);
-      rh = (uint32_t)f64_to_bf16_rne(db0 * t0.x + da0 * t0.y) | ((uint32_t)f64_to_bf16_rne(db1 * t1.x + da1 * t1.y) << 16);
-    }
-    lo[i] = rl;
-    hi[i] = rh;
-  }
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    if (pos[i] < 0) continue;
-    uint8_t* lo_p = lo_base + sw128_offset(row0 + i, lane >> 2);
-    *reinterpret_cast<uint32_t*>(lo_p) = lo[i];
-    *reinterpret_cast<uint32_t*>(lo_p + 16384) = hi[i];
   }
 }
 
@@ -278,8 +239,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       tma_prefetch_desc(&tm_qw);
       uint32_t cQ = 0, cK = 0, cV = 0;
       for (int item = pair_id; item < n_items; item += n_pairs) {
-        const int group = item / sch.ipg, within = item % sch.ipg;
-        const int c = group / prm.Hkv, hkv = group % prm.Hkv;
+        int group, within, c, hkv;
+        sch.d_ipg.divmod(item, group, within);
+        sch.d_hkv.divmod(group, c, hkv);
         const int nsub = n_subitems2(sch, within);
         for (int sub = 0; sub < nsub; ++sub) {
           const Blk bk = decode_blk(sch, rank, hkv, within, sub);
@@ -357,8 +319,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint32_t rk_u32 = smem_u32(cx.rK);
       uint32_t cQ = 0, cK = 0, cS = 0, cT = 0, n_done = 0;
       for (int item = pair_id; item < n_items; item += n_pairs) {
-        const int group = item / sch.ipg, within = item % sch.ipg;
-        const int hkv = group % prm.Hkv;
+        int group, within, c_unused, hkv;
+        sch.d_ipg.divmod(item, group, within);
+        sch.d_hkv.divmod(group, c_unused, hkv);
         const int nsub = n_subitems2(sch, within);
         for (int sub = 0; sub < nsub; ++sub) {
           const Blk bk = decode_blk(sch, rank, hkv, within, sub);
@@ -437,8 +400,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint32_t rv_u32 = smem_u32(cx.rV);
       uint32_t cS = 0, n_done = 0, n_turn = 0;
       for (int item = pair_id; item < n_items; item += n_pairs) {
-        const int group = item / sch.ipg, within = item % sch.ipg;
-        const int hkv = group % prm.Hkv;
+        int group, within, c_unused, hkv;
+        sch.d_ipg.divmod(item, group, within);
+        sch.d_hkv.divmod(group, c_unused, hkv);
         const int nsub = n_subitems2(sch, within);
         for (int sub = 0; sub < nsub; ++sub) {
           const Blk bk = decode_blk(sch, rank, hkv, within, sub);
@@ -483,22 +447,34 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint32_t cQ = 0, cS = 0, cT = 0, n_done = 0, n_tail = 0;
     uint32_t n_pub_mine = 0, n_pub_other = 0;                // publications made by this warpgroup / seen from the other
     bool pre_rotated = false;                                // the next block's Q is already rotated (cQ counts it)
+    // The output tile is stored from the block's Q buffer.  The thread that issued the store does not wait for
+    // it there (its warp would reach the next block's first tile a few thousand cycles after the others, and a
+    // tile is only as fast as its slowest warp): it waits, and hands the buffer back to the producer, after its
+    // first tile of the next block, when the store has long been read.
+    int store_pending = -1;                                  // thread 0: Q buffer of a store that may still be reading it
+    auto finish_store = [&]() {
+      if (tid == 0 && store_pending >= 0) {
+        tma_store_wait_read();
+        mbar_arrive(&mi.q_free[store_pending]);
+        store_pending = -1;
+      }
+    };
     auto rotate_q = [&](const Blk& b) {                      // RoPE of a Q tile in shared memory, half a row per thread
       const int qb = cQ & 1;
       WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
       ++cQ;
       {
         const int tok0 = b.t * TILE, L = prm.L;
-        rope_rows_warp(cx.sQ[qb], warp * 16, lane, prm.rope_tab, prm.rope_tab32,
-                       [=](int row) { return tok0 + row < L ? tok0 + row : -1; });
+        rope_rows_warp(cx.sQ[qb], warp * 16, lane, prm.rope_tab4, prm.rope_tab, [=](int row) { return tok0 + row < L ? tok0 + row : -1; });
       }
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.q_ready[qb], 0));
     };
     for (int item = pair_id; item < n_items; item += n_pairs) {
-      const int group = item / sch.ipg, within = item % sch.ipg;
-      const int c = group / prm.Hkv, hkv = group % prm.Hkv;
+      int group, within, c, hkv;
+      sch.d_ipg.divmod(item, group, within);
+      sch.d_hkv.divmod(group, c, hkv);
       const int nsub = n_subitems2(sch, within);
       for (int sub = 0; sub < nsub; ++sub) {
         const Blk bk = decode_blk(sch, rank, hkv, within, sub);
@@ -618,6 +594,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.p_b[hlf][sb], 0));
+          finish_store();
         }
         // the warpgroup that did not own the last tile consumes its owner's publication; then both
         // bring their partial sums to the final reference maximum
@@ -634,18 +611,20 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
         const float m_used = m_seen;
+        finish_store();                                      // before the rotation below waits for the Q after next
         // ---- rotate the next block's Q now, so that its first S tiles are computed under this block's
         // epilogue (not across a score sweep, whose window queries come next in the Q buffers)
         pre_rotated = false;
-        if (PC2_EARLY_ROT && !(within == 0 && sub == nsub - 1)) {
+        if (!(within == 0 && sub == nsub - 1)) {
           int n_item = item, n_within = within, n_sub = sub + 1, n_hkv = hkv;
           bool have = true;
           if (n_sub == nsub) {
             n_item = item + n_pairs;
             n_sub = 0;
             have = n_item < n_items;
-            n_within = n_item % sch.ipg;
-            n_hkv = (n_item / sch.ipg) % prm.Hkv;
+            int n_group, n_c;
+            sch.d_ipg.divmod(n_item, n_group, n_within);
+            sch.d_hkv.divmod(n_group, n_c, n_hkv);
           }
           if (have) {
             rotate_q(decode_blk(sch, rank, n_hkv, n_within, n_sub));
@@ -700,12 +679,12 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (bk.t * TILE < prm.L) {
             for (int a = 0; a < 2; ++a) tma_store_4d(&tm_o, myQ + a * 16384, a * 64, bk.h, bk.t * TILE, c);
             tma_store_commit();
-            tma_store_wait_read();
           }
-          mbar_arrive(&mi.q_free[qb]);
+          store_pending = qb;                                // released by finish_store() once the store has read it
         }
       }
       if (within == 0) {
+        finish_store();                                      // a later sweep pass loads window queries into that buffer
         // ---- score sweep.  First make the window rows' log-sum-exp of all heads visible in both CTAs.
         __syncwarp();
         if (lane == 0) {
@@ -720,8 +699,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           ++cQ;
           {
             const int w0 = prm.L - prm.w, ww = prm.w, nr = rows_half;
-            rope_rows_warp(cx.sQ[qb], warp * 16, lane, prm.rope_tab, prm.rope_tab32,
-                           [=](int row) { return row < nr ? w0 + (row % ww) : -1; });
+            rope_rows_warp(cx.sQ[qb], warp * 16, lane, prm.rope_tab4, prm.rope_tab, [=](int row) { return row < nr ? w0 + (row % ww) : -1; });
           }
           fence_proxy_async_smem();
           __syncwarp();
@@ -768,6 +746,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
     }
+    finish_store();
     if (tid == 0) tma_store_wait_all();
   }
 
@@ -787,12 +766,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 // maps: 0 q (box 64 x 128 tokens), 1 rotated keys (64 x 128), 2 v (64 x 128), 3 o (store), 4 q with a
 // w-token box, 5 rotated keys with a 64-token box.  The grid is a whole number of CTA pairs.
 cudaError_t launch_prefill_pair(const CUtensorMap* maps, const PrefillParams& prm, int sm_count, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(prefill_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  // the opt-in to large dynamic shared memory is a per-device attribute of the function: set it on every call
+  // (a host-side call of a few hundred nanoseconds) rather than remember which devices have it
+  if (cudaError_t e = cudaFuncSetAttribute(prefill_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES); e != cudaSuccess) return e;
   const int grid = (sm_count / 2) * 2;
   if (grid < 2) return cudaErrorInvalidConfiguration;
   if ((prm.Hq / prm.Hkv) % 2 != 0) return cudaErrorInvalidValue;   // the pair kernel takes even group sizes

@@ -3,10 +3,11 @@
 // fp64 and rounded once to bf16, so rotated keys are reproducible to the bit.
 #include "pc_kernels.h"
 #include "pc_sm100.cuh"
+#include "pc_rope_tile.cuh"
 
 namespace pc {
 
-__global__ void rope_table_kernel(double2* __restrict__ tab, float2* __restrict__ tab32, int n_pos, int half, double theta,
+__global__ void rope_table_kernel(double2* __restrict__ tab, float4* __restrict__ tab4, int n_pos, int half, double theta,
                                   int pos0) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_pos * half) return;
@@ -16,12 +17,15 @@ __global__ void rope_table_kernel(double2* __restrict__ tab, float2* __restrict_
   double s, c;
   sincos(phi, &s, &c);
   tab[i] = make_double2(c, s);
-  if (tab32 != nullptr) tab32[i] = make_float2((float)c, (float)s);   // the same entries rounded to fp32
+  if (tab4 != nullptr) {                                  // the same entries as fp32 head + fp32 tail: c = c_hi + c_lo to 2^-48
+    const float ch = (float)c, sh = (float)s;
+    tab4[i] = make_float4(ch, sh, (float)(c - (double)ch), (float)(s - (double)sh));
+  }
 }
 
-void launch_rope_table(double2* tab, float2* tab32, int n_pos, int d, double theta, int pos0, cudaStream_t st) {
+void launch_rope_table(double2* tab, float4* tab4, int n_pos, int d, double theta, int pos0, cudaStream_t st) {
   const int n = n_pos * (d / 2);
-  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, tab32, n_pos, d / 2, theta, pos0);
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, tab4, n_pos, d / 2, theta, pos0);
 }
 
 // One thread owns 8 consecutive pairs (t..t+7) of one position and walks all heads and a
@@ -72,6 +76,38 @@ void launch_rope_keys(const void* k, const long long k_stride[3], void* k_rot, c
   dim3 grid((unsigned)((n + 255) / 256), (unsigned)(C < 64 ? C : 64));
   rope_keys_kernel<<<grid, 256, 0, st>>>((const uint16_t*)k, k_stride[0], k_stride[1], k_stride[2], (uint16_t*)k_rot,
                                          tab, C, L, Hkv, d);
+}
+
+// RoPE of whole [128 rows x 128] tiles with the routine the attention kernel applies to its query tiles:
+// a tile is staged in shared memory in the 128-byte-swizzled layout the tensor cores read, rotated by eight
+// warps of 16 rows, and written back.  x, y: [C, L, H, 128] contiguous.
+__global__ void __launch_bounds__(256) rope_tiles_kernel(const uint4* __restrict__ x, uint4* __restrict__ y,
+                                                         const float4* __restrict__ tab4, const double2* __restrict__ tab,
+                                                         int L, int H, int tiles_per_chunk) {
+  __shared__ __align__(1024) uint8_t tile[32768];
+  const int tix = blockIdx.x % tiles_per_chunk, h = (blockIdx.x / tiles_per_chunk) % H, c = blockIdx.x / (tiles_per_chunk * H);
+  const int tok0 = tix * 128;
+  for (int i = threadIdx.x; i < 128 * 16; i += blockDim.x) {          // 16-byte pieces: row, piece (8 per 64-column atom)
+    const int row = i >> 4, piece = i & 15;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (tok0 + row < L) v = x[(((size_t)c * L + tok0 + row) * H + h) * 16 + piece];
+    *reinterpret_cast<uint4*>(tile + (piece >> 3) * 16384 + sw128_offset(row, piece & 7)) = v;
+  }
+  __syncthreads();
+  rope_rows_warp(tile, (threadIdx.x >> 5) * 16, threadIdx.x & 31, tab4, tab,
+                 [=](int row) { return tok0 + row < L ? tok0 + row : -1; });
+  __syncthreads();
+  for (int i = threadIdx.x; i < 128 * 16; i += blockDim.x) {
+    const int row = i >> 4, piece = i & 15;
+    if (tok0 + row < L)
+      y[(((size_t)c * L + tok0 + row) * H + h) * 16 + piece] =
+          *reinterpret_cast<const uint4*>(tile + (piece >> 3) * 16384 + sw128_offset(row, piece & 7));
+  }
+}
+
+void launch_rope_tiles(const void* x, void* y, const float4* tab4, const double2* tab, int C, int L, int H, cudaStream_t st) {
+  const int tiles = (L + 127) / 128;
+  rope_tiles_kernel<<<C * H * tiles, 256, 0, st>>>((const uint4*)x, (uint4*)y, tab4, tab, L, H, tiles);
 }
 
 }  // namespace pc

@@ -45,11 +45,11 @@ def test_status_strings_and_version(lib):
 
 def test_workspace_queries_are_host_only(lib):
     from paper_2502_14317_b200 import binding
-    # cfg1: 256 B counter + fp64 cos/sin table L * d/2 * 16 B + its fp32 copy L * d/2 * 8 B
-    assert binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128) == 256 + 8192 * 64 * 16 + 8192 * 64 * 8
-    assert binding.chunk_prefill_attn_workspace_bytes(4, 256, 16, 4, 2, 64) == 256 + 256 * 32 * 16 + 256 * 32 * 8
+    # cfg1: 256 B counter + fp64 cos/sin table L * d/2 * 16 B + its fp32 head+tail copy L * d/2 * 16 B
+    assert binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128) == 256 + 8192 * 64 * 16 + 8192 * 64 * 16
+    assert binding.chunk_prefill_attn_workspace_bytes(4, 256, 16, 4, 2, 64) == 256 + 256 * 32 * 16 + 256 * 32 * 16
     with_krot = binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128, k_rot_in_workspace=True)
-    assert with_krot == 256 + 8192 * 64 * 16 + 8192 * 64 * 8 + 16 * 8192 * 8 * 128 * 2
+    assert with_krot == 256 + 8192 * 64 * 16 + 8192 * 64 * 16 + 16 * 8192 * 8 * 128 * 2
     # unsupported shapes give 0
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 24, 4, 2, 64) == 0       # window not a power of two
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 2, 96) == 0       # head size
@@ -121,3 +121,23 @@ def test_reference_arm_other_ranks_do_nothing():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                        env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_launcher_makes_one_environment_per_gpu():
+    sys.path.insert(0, ROOT)
+    import bench
+    envs = bench.worker_environments(4, 29611, base_env={"KEEP": "1"})
+    assert len(envs) == 4 and all(e["KEEP"] == "1" for e in envs)
+    assert [e["RANK"] for e in envs] == ["0", "1", "2", "3"] == [e["LOCAL_RANK"] for e in envs]
+    assert {e["WORLD_SIZE"] for e in envs} == {"4"} and {e["MASTER_ADDR"] for e in envs} == {"127.0.0.1"}
+    assert {e["MASTER_PORT"] for e in envs} == {"29611"}
+
+
+def test_bench_without_launcher_starts_its_own_ranks():
+    # `bench.py --gpus 2` with no WORLD_SIZE in the environment must start two ranks itself; on the reference
+    # arm rank 1 exits at once and rank 0 would time the oracle, so a tiny stand-in command is spawned instead
+    sys.path.insert(0, ROOT)
+    import bench
+    code = "import os, sys; sys.exit(0 if os.environ['WORLD_SIZE'] == '2' and os.environ['RANK'] in '01' else 7)"
+    assert bench.spawn_workers([sys.executable, "-c", code], 2) == 0
+    assert bench.spawn_workers([sys.executable, "-c", "import os, sys; sys.exit(5 * int(os.environ['RANK']))"], 2) == 5

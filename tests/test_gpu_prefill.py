@@ -151,3 +151,26 @@ def test_argument_errors():
     rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), None, _ptr(k), _ptr(k), _ptr(o), None, None, _ptr(S), _ptr(Lw),
                                    None, _ptr(ws), ws.numel(), None)
     assert rc == -1                                                     # PC_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("C,L,H,d,theta", [
+    (2, 8192, 4, 128, 500000.0),           # the routine of the tile prologue, positions up to 8191 (angles up to 8191 rad)
+    (1, 4096, 8, 128, 10000.0),
+    (3, 333, 2, 128, 10000.0),             # ragged last tile
+    (2, 1000, 3, 64, 10000.0),             # head size 64: the fp64 pre-pass kernel
+])
+def test_rope_position_reuse_equals_fp64_rotation_rounded_once(C, L, H, d, theta):
+    """The query rotation of the tile prologue is fp32 with two exact fallbacks; its bits must be those of the
+    oracle's fp64 rotation.  Mixed magnitudes so that many outputs sit near a bf16 rounding boundary; with
+    millions of outputs the second level (about 1 in 4000) runs thousands of times."""
+    import paper_2502_14317_b200 as pc
+    rng = np.random.default_rng(5 + L + d)
+    x = rng.standard_normal((C, L, H, d)).astype(np.float32) * np.exp2(rng.integers(-6, 7, size=(C, L, H, 1))).astype(np.float32)
+    x[0, :, 0, : d // 2] = np.float32(1.0)                    # exact cosines / sines of the table reach the output
+    x[0, :, 0, d // 2:] = np.float32(0.0)
+    bits = pc_inputs.f32_to_bf16_bits(x)
+    got = to_bits(pc.rope_position_reuse(to_dev(bits), rope_theta=theta))
+    torch.cuda.synchronize()
+    ref = orc.rope_bf16(bits, theta)
+    bad = np.argwhere(got != ref)
+    assert bad.shape[0] == 0, f"{bad.shape[0]} of {ref.size} rotated values differ from the fp64 rotation, first at {bad[0]}"
