@@ -60,6 +60,10 @@ PC_API const char* pc_status_string(int32_t status);
 /* Library version, major * 1000 + minor. */
 PC_API int32_t pc_version(void);
 
+/* Number of kernels the library has launched in this process so far (all calls, all streams, all devices):
+ * the difference of two readings counts the launches in between.  Host-side counter, no GPU work. */
+PC_API uint64_t pc_launch_count(void);
+
 /* ------------------------------------------------------------------------------------
  * Chunk-local causal attention with position reuse and fused query-window scores.
  * Paper: Sec. 3.1 "Parallel attention" (chunking, Eq. 1-2) and "Parallel KV cache
@@ -99,9 +103,8 @@ PC_API int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q,
  *     y[c, p, h, :] = bf16( RoPE(x[c, p, h, :]) at position p ),  pairs (t, t + d/2),
  *     angle p * theta^(-2t/d), evaluated so that the result equals the fp64 rotation
  *     rounded once to bf16.
- * This is the rotation pc_chunk_prefill_attn applies to queries in its tile prologue and to
- * keys in its pre-pass (for d = 128 it runs the very routine of the tile prologue), offered
- * for callers that want rotated queries or keys as tensors.  x, y [C,L,H,d] bf16 contiguous.
+ * This is the pass pc_chunk_prefill_attn runs over its queries and keys before the attention
+ * kernel (same kernel), offered for callers that want rotated queries or keys as tensors.  x, y [C,L,H,d] bf16 contiguous.
  * Workspace: pc_rope_position_reuse_workspace_bytes(L, d) (cos/sin tables).
  */
 PC_API size_t pc_rope_position_reuse_workspace_bytes(int32_t L, int32_t d);

@@ -5,12 +5,14 @@
 #include "pc_kernels.h"
 #include "pc_tmap.h"
 
+#include <atomic>
 #include <cmath>
 #include <cstring>
 
-#ifndef PC_FORCE_SINGLE_CTA
-#define PC_FORCE_SINGLE_CTA 0
-#endif
+namespace pc {
+static std::atomic<unsigned long long> g_launches{0};
+void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+}  // namespace pc
 
 namespace {
 
@@ -47,14 +49,15 @@ void fill_strides(const int64_t in[3], int64_t out[3], int64_t tokens, int64_t h
 bool strides_ok(const int64_t s[3], int64_t d) { return s[0] > 0 && s[1] > 0 && s[2] >= d && s[0] % 8 == 0 && s[1] % 8 == 0 && s[2] % 8 == 0; }
 
 struct PrefillLayout {
-  size_t off_counter, off_table, off_table32, off_krot, total;
+  size_t off_counter, off_table, off_table32, off_qrot, off_krot, total;
 };
 PrefillLayout prefill_layout(const pc_prefill_desc* d, bool krot_in_ws) {
   PrefillLayout l;
   size_t off = 0;
   l.off_counter = off; off += ALIGN;
   l.off_table = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(double2));
-  l.off_table32 = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(float4));
+  l.off_table32 = off; off += align_up((size_t)d->L * (d->d / 2) * sizeof(float4));   // fp32 heads, then fp32 tails
+  l.off_qrot = off; off += align_up((size_t)d->C * d->L * d->Hq * d->d * 2);         // rotated queries
   l.off_krot = off;
   if (krot_in_ws) off += align_up((size_t)d->C * d->L * d->Hkv * d->d * 2);
   l.total = off;
@@ -89,7 +92,9 @@ const char* pc_status_string(int32_t status) {
   }
 }
 
-int32_t pc_version(void) { return 1000; }
+int32_t pc_version(void) { return 1001; }
+
+uint64_t pc_launch_count(void) { return pc::g_launches.load(std::memory_order_relaxed); }
 
 // ------------------------------------------------------------------------------------ prefill
 size_t pc_chunk_prefill_attn_workspace_bytes(const pc_prefill_desc* desc, int32_t k_rot_in_workspace) {
@@ -122,46 +127,48 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   int* counter = reinterpret_cast<int*>(ws + lay.off_counter);
   double2* table = reinterpret_cast<double2*>(ws + lay.off_table);
-  float4* table32 = reinterpret_cast<float4*>(ws + lay.off_table32);
+  float4* table_hi = reinterpret_cast<float4*>(ws + lay.off_table32);
+  float4* table_lo = table_hi + (size_t)desc->L * (d / 4);
   void* krot = krot_in_ws ? static_cast<void*>(ws + lay.off_krot) : k_rot;
+  void* qrot = ws + lay.off_qrot;
 
   // tensor maps (innermost first: d, head, token, chunk)
   CUtensorMap maps[6];
   const uint64_t q_dims[4] = {(uint64_t)d, (uint64_t)desc->Hq, (uint64_t)desc->L, (uint64_t)desc->C};
   const uint64_t kv_dims[4] = {(uint64_t)d, (uint64_t)desc->Hkv, (uint64_t)desc->L, (uint64_t)desc->C};
-  const uint64_t q_str[3] = {(uint64_t)qs[2], (uint64_t)qs[1], (uint64_t)qs[0]};
+  const uint64_t q_str[3] = {(uint64_t)d, (uint64_t)desc->Hq * d, (uint64_t)desc->L * desc->Hq * d};   // rotated queries: contiguous
   const uint64_t v_str[3] = {(uint64_t)vs[2], (uint64_t)vs[1], (uint64_t)vs[0]};
   const uint64_t o_str[3] = {(uint64_t)os[2], (uint64_t)os[1], (uint64_t)os[0]};
   const uint64_t kr_str[3] = {(uint64_t)d, (uint64_t)desc->Hkv * d, (uint64_t)desc->L * desc->Hkv * d};
   const uint32_t box_tile[4] = {64, 1, 128, 1};
   const uint32_t box_win[4] = {64, 1, (uint32_t)desc->w, 1};
   const uint32_t box_half[4] = {64, 1, 64, 1};
-  if (!pc::make_tmap_bf16_4d(&maps[0], q, q_dims, q_str, box_tile) ||
+  if (!pc::make_tmap_bf16_4d(&maps[0], qrot, q_dims, q_str, box_tile) ||
       !pc::make_tmap_bf16_4d(&maps[1], krot, kv_dims, kr_str, box_tile) ||
       !pc::make_tmap_bf16_4d(&maps[2], v, kv_dims, v_str, box_tile) ||
       !pc::make_tmap_bf16_4d(&maps[3], o, q_dims, o_str, box_tile) ||
-      !pc::make_tmap_bf16_4d(&maps[4], q, q_dims, q_str, box_win) ||
+      !pc::make_tmap_bf16_4d(&maps[4], qrot, q_dims, q_str, box_win) ||
       !pc::make_tmap_bf16_4d(&maps[5], krot, kv_dims, kr_str, box_half))
     return PC_ERR_CUDA;
 
   if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return PC_ERR_CUDA;
-  pc::launch_rope_table(table, table32, desc->L, d, (double)desc->rope_theta, 0, st);
-  const long long ks_ll[3] = {ks[0], ks[1], ks[2]};
-  pc::launch_rope_keys(k, ks_ll, krot, table, desc->C, desc->L, desc->Hkv, d, st);
+  pc::launch_rope_table(table, table_hi, table_lo, desc->L, d, (double)desc->rope_theta, 0, st);
+  // queries and keys are rotated once, ahead of the attention kernel (positions 0 .. L-1 in every chunk)
+  const long long ks_ll[3] = {ks[0], ks[1], ks[2]}, qs_ll[3] = {qs[0], qs[1], qs[2]};
+  pc::launch_rope_rows(k, ks_ll, krot, table, table_hi, table_lo, desc->C, desc->L, desc->Hkv, d, st);
+  pc::launch_rope_rows(q, qs_ll, qrot, table, table_hi, table_lo, desc->C, desc->L, desc->Hq, d, st);
 
   pc::PrefillParams prm;
   prm.C = desc->C; prm.L = desc->L; prm.w = desc->w; prm.Hq = desc->Hq; prm.Hkv = desc->Hkv;
   const double scale = desc->softmax_scale > 0.0f ? (double)desc->softmax_scale : 1.0 / std::sqrt((double)d);
   prm.scale_log2 = (float)(scale * 1.4426950408889634);
-  prm.rope_tab = table;
-  prm.rope_tab4 = table32;
   prm.lse = lse; prm.win_lse = win_lse; prm.win_score = win_score;
   prm.status = status_word; prm.counter = counter;
   // head size 128 with an even number of q-heads per kv-head runs on CTA pairs (cta_group::2: the two CTAs take
   // the same query tile of two heads that share K/V); head size 64 and odd group sizes (multi-head attention:
   // one q-head per kv-head) run on single CTAs with two query blocks each
   const bool even_group = ((desc->Hq / desc->Hkv) % 2) == 0;
-  const cudaError_t le = (d == 128 && even_group && dev.sm_count >= 2 && !PC_FORCE_SINGLE_CTA)
+  const cudaError_t le = (d == 128 && even_group && dev.sm_count >= 2)
                              ? pc::launch_prefill_pair(maps, prm, dev.sm_count, st)
                              : pc::launch_prefill_attn(maps, prm, d, dev.sm_count, st);
   if (le != cudaSuccess) return PC_ERR_CUDA;
@@ -185,14 +192,11 @@ int32_t pc_rope_position_reuse(const void* x, int32_t C, int32_t L, int32_t H, i
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   double2* table = reinterpret_cast<double2*>(ws);
-  float4* table4 = reinterpret_cast<float4*>(ws + align_up((size_t)L * (d / 2) * sizeof(double2)));
-  pc::launch_rope_table(table, table4, L, d, (double)rope_theta, 0, st);
-  if (d == 128) {
-    pc::launch_rope_tiles(x, y, table4, table, C, L, H, st);
-  } else {
-    const long long str[3] = {(long long)L * H * d, (long long)H * d, d};
-    pc::launch_rope_keys(x, str, y, table, C, L, H, d, st);
-  }
+  float4* table_hi = reinterpret_cast<float4*>(ws + align_up((size_t)L * (d / 2) * sizeof(double2)));
+  float4* table_lo = table_hi + (size_t)L * (d / 4);
+  pc::launch_rope_table(table, table_hi, table_lo, L, d, (double)rope_theta, 0, st);
+  const long long str[3] = {(long long)L * H * d, (long long)H * d, d};
+  pc::launch_rope_rows(x, str, y, table, table_hi, table_lo, C, L, H, d, st);
   return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
 }
 
@@ -419,7 +423,7 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
     return PC_ERR_CUDA;
 
   if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return PC_ERR_CUDA;
-  pc::launch_rope_table(table, nullptr, w, d, (double)rope_theta, q_pos0, st);
+  pc::launch_rope_table(table, nullptr, nullptr, w, d, (double)rope_theta, q_pos0, st);
 
   pc::ParallelParams prm;
   prm.B = B; prm.w = w; prm.Hq = Hq; prm.Hkv = Hkv; prm.Nk = Nk;

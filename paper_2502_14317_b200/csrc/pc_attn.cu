@@ -358,7 +358,7 @@ __device__ __forceinline__ void turn_pass(const Ctx& cx, Waits& wt, int b) {
 // walks the ring, takes its turns and releases the stages it does not use, so that both
 // issuers arrive once on every kv_free barrier and the token keeps alternating.
 template <int D>
-__device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b, bool has_b, int nb_b, int n) {
+__device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b, bool has_b, int nb_b, int n, bool q_rotated_here) {
   using C = Cfg<D>;
   Misc& mi = *cx.mi;
   const uint32_t ring_u32 = smem_u32(cx.ring);
@@ -369,7 +369,9 @@ __device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b,
     mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
 #pragma unroll
     for (int e = 0; e < 2; ++e) mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
-    mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT);
+    // the query block is ready: rotated in shared memory by the softmax group (parallel attention), or, already
+    // rotated in global memory, as soon as its copy has landed (chunk prefill)
+    mbar_wait(q_rotated_here ? &mi.q_rot[b] : &mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT);
     ++wt.q[b];
   }
   {  // S(0)
@@ -555,7 +557,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const bool has_b = (b == 0) || it.hB >= 0;
           const int nb_b = (b == 0) ? it.tA + 1 : (it.hB >= 0 ? it.tB + 1 : 0);
           const int n = (it.hB >= 0 ? it.tB : it.tA) + 1;
-          mma_flash_block<D>(cx, wt, b, has_b, nb_b, n);
+          mma_flash_block<D>(cx, wt, b, has_b, nb_b, n, false);
         }
         if (within == 0) {
           // ---- score sweep: this issuer computes the columns of its own block (window rows b*128..)
@@ -564,7 +566,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
             const int rows_total = heads * prm.w;
             const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
-            if (rows_b > 0) { mbar_wait(&mi.q_rot[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
+            if (rows_b > 0) { mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
             for (int j = 0; j < sch.T; ++j) {
               const int e = j & 1;
               mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
@@ -595,7 +597,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t tS = cx.tmem + b * 128 + lane_sel, tO = cx.tmem + 256 + b * 128 + lane_sel;
     const float scale_log2 = prm.scale_log2;
     uint8_t* const myQ = b ? cx.sQ[1] : cx.sQ[0];
-    uint32_t n_q = 0, n_s = 0, n_o = 0, n_t0 = 0, n_t1 = 0;   // barrier use counts of this group
+    uint32_t n_s = 0, n_o = 0, n_t0 = 0, n_t1 = 0;            // barrier use counts of this group
     while (true) {
       const int item = consumer_next_item(cx, wt);
       if (item == ITEM_DONE) break;
@@ -607,12 +609,6 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int h = b ? it.hB : it.hA, t = b ? it.tB : it.tA;
         if (h < 0) continue;
         const int token = t * TILE + r;
-        // ---- Q prologue: rotate this thread's row in shared memory
-        mbar_wait(&mi.q_full[b], full_par(n_q), cx.abort_flag, cx.status, W_QFULL);
-        ++n_q;
-        if (token < prm.L) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)token * (D / 2));
-        fence_proxy_async_smem();
-        mbar_arrive(&mi.q_rot[b]);
         // ---- main loop over key tiles (causal: keys <= token; only the diagonal tile is masked)
         float m_used, l_run;
         const int n = t + 1;
@@ -663,13 +659,6 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
           const int rows_total = heads * prm.w;
           const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
-          if (rows_b > 0) {
-            mbar_wait(&mi.q_full[b], full_par(n_q), cx.abort_flag, cx.status, W_QFULL);
-            ++n_q;
-            if (r < rows_b) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)(prm.L - prm.w + (r % prm.w)) * (D / 2));
-            fence_proxy_async_smem();
-            mbar_arrive(&mi.q_rot[b]);
-          }
           const float* lse_rows = mi.lse2 + u * Gs * prm.w + b * TILE;   // log-sum-exp of the window row on column n
           for (int j = 0; j < sch.T; ++j) {
             const int e = j & 1;
@@ -820,7 +809,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
         if (item == ITEM_DONE) break;
         const Dec d = decode(item);
         const bool has_b = d.rows[b] > 0;
-        mma_flash_block<D>(cx, wt, b, has_b, has_b ? d.n : 0, d.n);
+        mma_flash_block<D>(cx, wt, b, has_b, has_b ? d.n : 0, d.n, true);
       }
     }
     __syncwarp();
@@ -947,6 +936,7 @@ static cudaError_t launch_prefill_t(const CUtensorMap* maps, const PrefillParams
   // (a host-side call of a few hundred nanoseconds) rather than remember which devices have it
   if (cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Cfg<D>::SMEM_BYTES); e != cudaSuccess) return e;
+  note_launch();
   prefill_attn_kernel<D><<<grid, NUM_THREADS, Cfg<D>::SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
   return cudaGetLastError();
 }
@@ -961,11 +951,13 @@ static cudaError_t launch_parallel_t(const CUtensorMap* maps, const ParallelPara
   // (a host-side call of a few hundred nanoseconds) rather than remember which devices have it
   if (cudaError_t e = cudaFuncSetAttribute(parallel_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Cfg<D>::SMEM_BYTES); e != cudaSuccess) return e;
+  note_launch();
   parallel_attn_kernel<D><<<grid, NUM_THREADS, Cfg<D>::SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (prm.n_split > 1) {
     const int rows = prm.B * prm.Hq * prm.w;
+    note_launch();
     parallel_merge_kernel<D><<<(rows + 7) / 8, 256, 0, st>>>(prm.part_o, prm.part_ml, prm.B * prm.Hq, prm.w, prm.Hq,
                                                             prm.n_split, prm.out, prm.lse_out);
     e = cudaGetLastError();

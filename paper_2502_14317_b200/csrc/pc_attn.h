@@ -10,8 +10,6 @@ namespace pc {
 struct PrefillParams {
   int C, L, w, Hq, Hkv;
   float scale_log2;              // softmax scale * log2(e)
-  const double2* rope_tab;       // [L][d/2] (cos, sin)
-  const float4* rope_tab4;       // the same entries as (cos_hi, sin_hi, cos_lo, sin_lo): fp32 head + tail
   float* lse;                    // [C,Hq,L] or null
   float* win_lse;                // [C,Hq,w]
   float* win_score;              // [C,Hkv,L]
@@ -19,7 +17,7 @@ struct PrefillParams {
   int* counter;                  // work-queue counter, zeroed before launch
 };
 
-// maps: q (box 64x1x128x1), k_rot, v, o (store), q with a w-row box
+// maps: rotated q (box 64x1x128x1), k_rot, v, o (store), rotated q with a w-row box
 cudaError_t launch_prefill_attn(const CUtensorMap* maps, const PrefillParams& prm, int d, int grid, cudaStream_t st);
 
 // Head size 128: CTA-pair kernel (pc_prefill2.cu).  maps as above plus maps[5] = rotated keys with a 64-token box.

@@ -6,17 +6,19 @@
 
 namespace pc {
 
-// ---- pc_rope.cu
-// cos/sin table: tab[p * (d/2) + t] = (cos, sin)(  (pos0 + p) * theta^(-2t/d) ), fp64; tab4 (may be null): the
-// same entries as (cos_hi, sin_hi, cos_lo, sin_lo), fp32 head + fp32 tail of each value.
-void launch_rope_table(double2* tab, float4* tab4, int n_pos, int d, double theta, int pos0, cudaStream_t st);
-// k_rot[c,p,h,:] = bf16( RoPE(k[c,p,h,:], position p) ), rotation evaluated in fp64.
-void launch_rope_keys(const void* k, const long long k_stride[3], void* k_rot, const double2* tab, int C, int L,
-                      int Hkv, int d, cudaStream_t st);
+// ---- pc_api.cu
+// Every kernel launch of the library is counted here (see pc_launch_count in pc.h).
+void note_launch();
 
-// y[c,p,h,:] = bf16( RoPE(x[c,p,h,:], position p) ) for head size 128, tile by tile with the routine of the
-// attention kernel's query prologue (fp32 with exact fallbacks: same bits as the fp64 rotation).
-void launch_rope_tiles(const void* x, void* y, const float4* tab4, const double2* tab, int C, int L, int H, cudaStream_t st);
+// ---- pc_rope.cu
+// cos/sin table: tab[p * (d/2) + t] = (cos, sin)(  (pos0 + p) * theta^(-2t/d) ), fp64; tab_hi, tab_lo (may be null): the
+// same entries split into an fp32 head and an fp32 tail (value = head + tail to 2^-48), one float4 per two pairs:
+// (cos_2i, cos_2i+1, sin_2i, sin_2i+1).
+void launch_rope_table(double2* tab, float4* tab_hi, float4* tab_lo, int n_pos, int d, double theta, int pos0, cudaStream_t st);
+// y[c,p,h,:] = bf16( RoPE(x[c,p,h,:], position p) ), the fp64 rotation rounded once; x addressed by element strides
+// (chunk, token, head), y contiguous [C,L,H,d].
+void launch_rope_rows(const void* x, const long long x_stride[3], void* y, const double2* tab, const float4* tab_hi,
+                      const float4* tab_lo, int C, int L, int H, int d, cudaStream_t st);
 
 // ---- pc_select_gather.cu
 void launch_chunk_score(const float* win_lse, int C, int n_per_chunk, float* score, cudaStream_t st);

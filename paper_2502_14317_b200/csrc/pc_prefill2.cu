@@ -15,8 +15,8 @@
 // may run into the same buffer, so that S is waiting when the warpgroup comes back; P(j) goes to
 // the warpgroup's P buffer once P V of its previous tile has run.
 //
-// Warps (12 per CTA): 0-3 softmax of even tiles, 4-7 softmax of odd tiles (both: Q rotation,
-// epilogue and score sweep split by halves),
+// Warps (12 per CTA): 0-3 softmax of even tiles, 4-7 softmax of odd tiles (both: epilogue and score
+// sweep split by halves),
 // 8 TMA producer, 9 issuer of Q K^T, 10 and 11 issuers of P V for even / odd tiles (issuers run in
 // the leader CTA only).  Several issuers because a tcgen05.mma issue blocks while the pipe is busy
 // and every barrier wait or commit of an issuing thread costs it about a hundred cycles.
@@ -28,7 +28,6 @@
 #include "pc_kernels.h"
 #include "pc_attn.h"
 #include "pc_sm100.cuh"
-#include "pc_rope_tile.cuh"
 
 namespace pc {
 
@@ -46,11 +45,11 @@ constexpr int Q_BYTES = 32768;
 constexpr uint32_t TM_O = 384;               // accumulator columns
 constexpr float LAZY_RESCALE = 8.0f;         // log2 units
 
-enum { W2_QFULL = 201, W2_QREADY, W2_QFREE, W2_KFULL, W2_KFREE, W2_VFULL, W2_VFREE, W2_SFULL, W2_PA, W2_PB,
+enum { W2_QFULL = 201, W2_QFREE, W2_KFULL, W2_KFREE, W2_VFULL, W2_VFREE, W2_SFULL, W2_PA, W2_PB,
        W2_PVDONE, W2_OFULL, W2_ACCFREE, W2_LSE, W2_TFULL, W2_TFREE, W2_MPUB, W2_TURN };
 
 struct __align__(16) Misc2 {
-  uint64_t q_full[2], q_ready[2], q_free[2];
+  uint64_t q_full[2], q_free[2];             // q_full: leader only, counts the bytes of both CTAs' query tiles
   uint64_t k_full[NKS], k_free[NKS], v_full[NVS], v_free[NVS];
   uint64_t s_full[2][NSB];                   // [owning warpgroup][buffer]: a waiter must see every phase of its barrier
   uint64_t p_a[2][NSB], p_b[2][NSB];         // [owning warpgroup = P V issuer][buffer]
@@ -173,7 +172,7 @@ __device__ __forceinline__ void mbar_wait_cluster(uint64_t* bar, uint32_t parity
 
 __device__ __forceinline__ void init_barriers2(Misc2& mi) {
   for (int b = 0; b < 2; ++b) {
-    mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_ready[b], 16); mbar_init(&mi.q_free[b], 1);
+    mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_free[b], 1);
     mbar_init(&mi.t_full[b], 1); mbar_init(&mi.t_free[b], 16);
   }
   for (int s = 0; s < NKS; ++s) { mbar_init(&mi.k_full[s], 1); mbar_init(&mi.k_free[s], 1); }
@@ -248,8 +247,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           {
             const int qb = cQ & 1;
             WAIT2(&mi.q_free[qb], free_par(cQ >> 1), W2_QFREE);
-            mbar_arrive_expect_tx(&mi.q_full[qb], Q_BYTES);
-            for (int a = 0; a < 2; ++a) tma_load_4d(cx.sQ[qb] + a * 16384, &tm_q, &mi.q_full[qb], a * 64, bk.h, bk.t * TILE, c);
+            if (leader) mbar_arrive_expect_tx(&mi.q_full[qb], 2 * Q_BYTES);
+            const uint32_t bar = map_to_cta(&mi.q_full[qb], 0);
+            for (int a = 0; a < 2; ++a) tma_load_4d_pair(cx.sQ[qb] + a * 16384, &tm_q, bar, a * 64, bk.h, bk.t * TILE, c);
             ++cQ;
           }
           for (int j = 0; j < bk.n; ++j) {
@@ -276,13 +276,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int u = 0; u < sch.n_pass; ++u) {
             const int qb = cQ & 1;
             WAIT2(&mi.q_free[qb], free_par(cQ >> 1), W2_QFREE);
-            mbar_arrive_expect_tx(&mi.q_full[qb], rows_half * D * 2);
+            if (leader) mbar_arrive_expect_tx(&mi.q_full[qb], 2 * rows_half * D * 2);
+            const uint32_t bar = map_to_cta(&mi.q_full[qb], 0);
             for (int i = 0; i < sch.hp; ++i) {
               int g = u * 2 * sch.hp + (int)rank * sch.hp + i;
               if (g >= sch.G) g = sch.G - 1;              // filler rows: loaded, never summed
               for (int a = 0; a < 2; ++a)
-                tma_load_4d(cx.sQ[qb] + a * 16384 + i * prm.w * 128, &tm_qw, &mi.q_full[qb], a * 64, hkv * sch.G + g,
-                            prm.L - prm.w, c);
+                tma_load_4d_pair(cx.sQ[qb] + a * 16384 + i * prm.w * 128, &tm_qw, bar, a * 64, hkv * sch.G + g,
+                                 prm.L - prm.w, c);
             }
             ++cQ;
             if (cK & 1) {                                 // a full key tile takes an even-aligned pair of stages
@@ -326,7 +327,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         for (int sub = 0; sub < nsub; ++sub) {
           const Blk bk = decode_blk(sch, rank, hkv, within, sub);
           const int qb = cQ & 1;
-          WAIT2(&mi.q_ready[qb], full_par(cQ >> 1), W2_QREADY);
+          WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);           // the query tiles of both CTAs have landed
           ++cQ;
           const uint32_t q_u32 = smem_u32(cx.sQ[qb]);
           for (int j = 0; j < bk.n; ++j) {
@@ -354,7 +355,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           WAIT2(&mi.acc_free, free_par(n_done), W2_ACCFREE);
           for (int u = 0; u < sch.n_pass; ++u) {
             const int qb = cQ & 1;
-            WAIT2(&mi.q_ready[qb], full_par(cQ >> 1), W2_QREADY);
+            WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
             ++cQ;
             const uint32_t q_u32 = smem_u32(cx.sQ[qb]);
             if (cK & 1) {
@@ -446,7 +447,6 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t a_acc_free = map_to_cta(&mi.acc_free, 0);
     uint32_t cQ = 0, cS = 0, cT = 0, n_done = 0, n_tail = 0;
     uint32_t n_pub_mine = 0, n_pub_other = 0;                // publications made by this warpgroup / seen from the other
-    bool pre_rotated = false;                                // the next block's Q is already rotated (cQ counts it)
     // The output tile is stored from the block's Q buffer.  The thread that issued the store does not wait for
     // it there (its warp would reach the next block's first tile a few thousand cycles after the others, and a
     // tile is only as fast as its slowest warp): it waits, and hands the buffer back to the producer, after its
@@ -459,18 +459,6 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         store_pending = -1;
       }
     };
-    auto rotate_q = [&](const Blk& b) {                      // RoPE of a Q tile in shared memory, half a row per thread
-      const int qb = cQ & 1;
-      WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
-      ++cQ;
-      {
-        const int tok0 = b.t * TILE, L = prm.L;
-        rope_rows_warp(cx.sQ[qb], warp * 16, lane, prm.rope_tab4, prm.rope_tab, [=](int row) { return tok0 + row < L ? tok0 + row : -1; });
-      }
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.q_ready[qb], 0));
-    };
     for (int item = pair_id; item < n_items; item += n_pairs) {
       int group, within, c, hkv;
       sch.d_ipg.divmod(item, group, within);
@@ -479,8 +467,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int sub = 0; sub < nsub; ++sub) {
         const Blk bk = decode_blk(sch, rank, hkv, within, sub);
         const int token = bk.t * TILE + r;
-        if (!pre_rotated) rotate_q(bk);                      // usually done at the end of the previous block
-        const int qb = (cQ - 1) & 1;
+        const int qb = cQ & 1;                               // this block's query buffer (its output is staged there)
+        ++cQ;
         uint8_t* const myQ = cx.sQ[qb];
         // ---- key tiles: the two warpgroups take alternate tiles (whole rows, one thread per row), so the
         // load / maximum phase of one tile runs under the exponentials of the other.  The running
@@ -611,26 +599,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
         const float m_used = m_seen;
-        finish_store();                                      // before the rotation below waits for the Q after next
-        // ---- rotate the next block's Q now, so that its first S tiles are computed under this block's
-        // epilogue (not across a score sweep, whose window queries come next in the Q buffers)
-        pre_rotated = false;
-        if (!(within == 0 && sub == nsub - 1)) {
-          int n_item = item, n_within = within, n_sub = sub + 1, n_hkv = hkv;
-          bool have = true;
-          if (n_sub == nsub) {
-            n_item = item + n_pairs;
-            n_sub = 0;
-            have = n_item < n_items;
-            int n_group, n_c;
-            sch.d_ipg.divmod(n_item, n_group, n_within);
-            sch.d_hkv.divmod(n_group, n_c, n_hkv);
-          }
-          if (have) {
-            rotate_q(decode_blk(sch, rank, n_hkv, n_within, n_sub));
-            pre_rotated = true;
-          }
-        }
+        finish_store();
         // ---- epilogue: combine the two half-row sums, normalise, stage bf16 rows in this block's
         // (now idle) Q buffer, TMA store
         WAIT2(&mi.o_full, full_par(n_done), W2_OFULL);
@@ -694,16 +663,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_wait_cluster(&mi.lse_ready, full_par(n_tail), cx.abort_flag, cx.status, W2_LSE);
         ++n_tail;
         for (int u = 0; u < sch.n_pass; ++u) {
-          const int qb = cQ & 1;
-          WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
+          const int qb = cQ & 1;                             // window queries of this pass (loaded and consumed by other warps)
           ++cQ;
-          {
-            const int w0 = prm.L - prm.w, ww = prm.w, nr = rows_half;
-            rope_rows_warp(cx.sQ[qb], warp * 16, lane, prm.rope_tab4, prm.rope_tab, [=](int row) { return row < nr ? w0 + (row % ww) : -1; });
-          }
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.q_ready[qb], 0));
           // this thread sums the columns of the heads that CTA `hlf` loaded: local head i = ncol / w
           const int g_base = u * 2 * sch.hp + hlf * sch.hp;
           for (int jj = 0; jj < n_sweep_tiles; ++jj) {
@@ -772,6 +733,7 @@ cudaError_t launch_prefill_pair(const CUtensorMap* maps, const PrefillParams& pr
   const int grid = (sm_count / 2) * 2;
   if (grid < 2) return cudaErrorInvalidConfiguration;
   if ((prm.Hq / prm.Hkv) % 2 != 0) return cudaErrorInvalidValue;   // the pair kernel takes even group sizes
+  note_launch();
   prefill_pair_kernel<<<grid, NT2, SMEM2_BYTES, st>>>(maps[0], maps[5], maps[1], maps[2], maps[3], maps[4], prm);
   return cudaGetLastError();
 }

@@ -24,6 +24,7 @@ __global__ void queue_init_kernel(float* q_score, int* q_chunk, int m) {
 }
 
 void launch_queue_init(float* q_score, int* q_chunk, int m, cudaStream_t st) {
+  note_launch();
   queue_init_kernel<<<1, 256, 0, st>>>(q_score, q_chunk, m);
 }
 
@@ -81,6 +82,7 @@ __global__ void __launch_bounds__(QUEUE_MAX) queue_update_kernel(const float* __
 
 void launch_queue_update(const float* score, int Cb, int chunk_id0, int lower_is_better, int m, float* q_score,
                          int* q_chunk, int* slot_src, cudaStream_t st) {
+  note_launch();
   queue_update_kernel<<<1, QUEUE_MAX, 0, st>>>(score, Cb, chunk_id0, lower_is_better, m, q_score, q_chunk, slot_src);
 }
 
@@ -136,12 +138,14 @@ __global__ void __launch_bounds__(256) queue_emit_kernel(const uint4* __restrict
 cudaError_t launch_queue_emit(const int* q_chunk, int m, int Hkv, int k, int d, const void* q_k, const void* q_v,
                               const int* q_pos, int* kept_out, int* slot_order, void* k_out, void* v_out, int* pos_out,
                               int sm_count, cudaStream_t st) {
+  note_launch();
   queue_order_kernel<<<1, QUEUE_MAX, 0, st>>>(q_chunk, m, kept_out, slot_order);
   const long long n_rows = (long long)Hkv * m * k;
   const int lpr = d / 8;
   const long long want = (n_rows * lpr + 255) / 256;
   int blocks = (int)(want < (long long)sm_count * 8 ? want : (long long)sm_count * 8);
   if (blocks < 1) blocks = 1;
+  note_launch();
   if (d == 128)
     queue_emit_kernel<128><<<blocks, 256, 0, st>>>((const uint4*)q_k, (const uint4*)q_v, q_pos, slot_order, m, Hkv, k,
                                                    (uint4*)k_out, (uint4*)v_out, pos_out);

@@ -1,113 +1,87 @@
 // RoPE with position reuse (Sec. 3.1 "Parallel attention": positions restart in every
-// chunk).  Pairs (t, t + d/2), angle p * theta^(-2t/d).  The rotation is evaluated in
-// fp64 and rounded once to bf16, so rotated keys are reproducible to the bit.
+// chunk).  Pairs (t, t + d/2), angle p * theta^(-2t/d).  Queries and keys are rotated once,
+// before the attention kernel, by a bandwidth-bound pass: the result is the fp64 rotation
+// rounded once to bf16 (see pc_rope_exact.cuh for how fp32 arithmetic gets there), so rotated
+// keys - an output that the gather copies - are reproducible to the bit.
 #include "pc_kernels.h"
-#include "pc_sm100.cuh"
-#include "pc_rope_tile.cuh"
+#include "pc_rope_exact.cuh"
 
 namespace pc {
 
-__global__ void rope_table_kernel(double2* __restrict__ tab, float4* __restrict__ tab4, int n_pos, int half, double theta,
-                                  int pos0) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n_pos * half) return;
-  const int p = i / half, t = i % half;
-  const double inv_freq = pow(theta, -2.0 * (double)t / (double)(2 * half));
-  const double phi = (double)(pos0 + p) * inv_freq;
-  double s, c;
-  sincos(phi, &s, &c);
-  tab[i] = make_double2(c, s);
-  if (tab4 != nullptr) {                                  // the same entries as fp32 head + fp32 tail: c = c_hi + c_lo to 2^-48
-    const float ch = (float)c, sh = (float)s;
-    tab4[i] = make_float4(ch, sh, (float)(c - (double)ch), (float)(s - (double)sh));
+// tab: (cos, sin) per (position, pair), fp64.  tab_hi / tab_lo: fp32 heads / tails of the same values, one float4
+// per two consecutive pairs (cos_2i, cos_2i+1, sin_2i, sin_2i+1); value = head + tail to 2^-48.
+__global__ void rope_table_kernel(double2* __restrict__ tab, float4* __restrict__ tab_hi, float4* __restrict__ tab_lo, int n_pos,
+                                  int half, double theta, int pos0) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;      // one thread per two pairs
+  if (i >= n_pos * (half / 2)) return;
+  const int p = i / (half / 2), t = 2 * (i % (half / 2));
+  double c[2], s[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const double inv_freq = pow(theta, -2.0 * (double)(t + e) / (double)(2 * half));
+    sincos((double)(pos0 + p) * inv_freq, &s[e], &c[e]);
+    tab[(size_t)p * half + t + e] = make_double2(c[e], s[e]);
+  }
+  if (tab_hi != nullptr) {
+    const float c0 = (float)c[0], c1 = (float)c[1], s0 = (float)s[0], s1 = (float)s[1];
+    tab_hi[i] = make_float4(c0, c1, s0, s1);
+    tab_lo[i] = make_float4((float)(c[0] - (double)c0), (float)(c[1] - (double)c1), (float)(s[0] - (double)s0),
+                            (float)(s[1] - (double)s1));
   }
 }
 
-void launch_rope_table(double2* tab, float4* tab4, int n_pos, int d, double theta, int pos0, cudaStream_t st) {
-  const int n = n_pos * (d / 2);
-  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, tab4, n_pos, d / 2, theta, pos0);
+void launch_rope_table(double2* tab, float4* tab_hi, float4* tab_lo, int n_pos, int d, double theta, int pos0, cudaStream_t st) {
+  const int n = n_pos * (d / 4);
+  note_launch();
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, tab_hi, tab_lo, n_pos, d / 2, theta, pos0);
 }
 
-// One thread owns 8 consecutive pairs (t..t+7) of one position and walks all heads and a
-// slice of chunks, so its 8 table entries are read once.
-__global__ void __launch_bounds__(256) rope_keys_kernel(const uint16_t* __restrict__ k, long long s_chunk,
-                                                        long long s_tok, long long s_head,
-                                                        uint16_t* __restrict__ k_rot, const double2* __restrict__ tab,
-                                                        int C, int L, int Hkv, int d) {
+// y[c,p,h,:] = bf16( RoPE(x[c,p,h,:], position p) ).  One thread owns 8 consecutive pairs (t .. t+7) of one
+// position and walks all heads and a slice of the chunks, so its table entries are read once and stay in
+// registers.  A warp covers 32 / (d/16) positions: every 16-byte access of a warp falls into fully used
+// 128-byte segments.
+__global__ void __launch_bounds__(256, 4) rope_rows_kernel(const uint16_t* __restrict__ x, long long s_chunk, long long s_tok,
+                                                           long long s_head, uint16_t* __restrict__ y,
+                                                           const float4* __restrict__ tab_hi, const float4* __restrict__ tab_lo,
+                                                           const double2* __restrict__ tab, int C, int L, int H, int d) {
   const int half = d / 2;
   const int groups = half / 8;                              // 16-byte groups per half row
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= (long long)L * groups) return;
   const int p = (int)(gid / groups), g = (int)(gid % groups);
-  double2 cs[8];
+  const size_t e0 = (size_t)p * half + g * 8;               // first pair of this thread in the tables
+  float4 hi[4];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) cs[i] = tab[(size_t)p * half + g * 8 + i];
+  for (int i = 0; i < 4; ++i) hi[i] = __ldg(tab_hi + e0 / 2 + i);
   for (int c = blockIdx.y; c < C; c += gridDim.y) {
-    for (int h = 0; h < Hkv; ++h) {
-      const uint16_t* src = k + (long long)c * s_chunk + (long long)p * s_tok + (long long)h * s_head;
-      uint16_t* dst = k_rot + (((size_t)c * L + p) * Hkv + h) * d;
-      const uint4 lo = *reinterpret_cast<const uint4*>(src + g * 8);
-      const uint4 hi = *reinterpret_cast<const uint4*>(src + half + g * 8);
-      const uint32_t lo_w[4] = {lo.x, lo.y, lo.z, lo.w}, hi_w[4] = {hi.x, hi.y, hi.z, hi.w};
-      uint32_t out_lo[4], out_hi[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        uint32_t rl = 0, rh = 0;
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const double x1 = (double)__uint_as_float(((lo_w[i] >> (16 * e)) & 0xFFFFu) << 16);
-          const double x2 = (double)__uint_as_float(((hi_w[i] >> (16 * e)) & 0xFFFFu) << 16);
-          const double2 t = cs[2 * i + e];
-          rl |= (uint32_t)f64_to_bf16_rne(x1 * t.x - x2 * t.y) << (16 * e);
-          rh |= (uint32_t)f64_to_bf16_rne(x2 * t.x + x1 * t.y) << (16 * e);
-        }
-        out_lo[i] = rl;
-        out_hi[i] = rh;
-      }
-      *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(out_lo[0], out_lo[1], out_lo[2], out_lo[3]);
-      *reinterpret_cast<uint4*>(dst + half + g * 8) = make_uint4(out_hi[0], out_hi[1], out_hi[2], out_hi[3]);
+    const uint16_t* src_c = x + (long long)c * s_chunk + (long long)p * s_tok + g * 8;
+    uint16_t* dst_c = y + ((size_t)c * L + p) * H * d + g * 8;
+#pragma unroll 1
+    for (int h = 0; h < H; ++h) {
+      const uint16_t* src = src_c + (long long)h * s_head;
+      uint16_t* dst = dst_c + (size_t)h * d;
+      const uint4 x1 = __ldg(reinterpret_cast<const uint4*>(src));
+      const uint4 x2 = __ldg(reinterpret_cast<const uint4*>(src + half));
+      uint4 y1, y2;
+      rope_two_pairs(x1.x, x2.x, hi[0], tab_lo + e0 / 2 + 0, tab + e0 + 0, y1.x, y2.x);
+      rope_two_pairs(x1.y, x2.y, hi[1], tab_lo + e0 / 2 + 1, tab + e0 + 2, y1.y, y2.y);
+      rope_two_pairs(x1.z, x2.z, hi[2], tab_lo + e0 / 2 + 2, tab + e0 + 4, y1.z, y2.z);
+      rope_two_pairs(x1.w, x2.w, hi[3], tab_lo + e0 / 2 + 3, tab + e0 + 6, y1.w, y2.w);
+      *reinterpret_cast<uint4*>(dst) = y1;
+      *reinterpret_cast<uint4*>(dst + half) = y2;
     }
   }
 }
 
-void launch_rope_keys(const void* k, const long long k_stride[3], void* k_rot, const double2* tab, int C, int L,
-                      int Hkv, int d, cudaStream_t st) {
+void launch_rope_rows(const void* x, const long long x_stride[3], void* y, const double2* tab, const float4* tab_hi,
+                      const float4* tab_lo, int C, int L, int H, int d, cudaStream_t st) {
   const long long n = (long long)L * (d / 16);
-  dim3 grid((unsigned)((n + 255) / 256), (unsigned)(C < 64 ? C : 64));
-  rope_keys_kernel<<<grid, 256, 0, st>>>((const uint16_t*)k, k_stride[0], k_stride[1], k_stride[2], (uint16_t*)k_rot,
-                                         tab, C, L, Hkv, d);
-}
-
-// RoPE of whole [128 rows x 128] tiles with the routine the attention kernel applies to its query tiles:
-// a tile is staged in shared memory in the 128-byte-swizzled layout the tensor cores read, rotated by eight
-// warps of 16 rows, and written back.  x, y: [C, L, H, 128] contiguous.
-__global__ void __launch_bounds__(256) rope_tiles_kernel(const uint4* __restrict__ x, uint4* __restrict__ y,
-                                                         const float4* __restrict__ tab4, const double2* __restrict__ tab,
-                                                         int L, int H, int tiles_per_chunk) {
-  __shared__ __align__(1024) uint8_t tile[32768];
-  const int tix = blockIdx.x % tiles_per_chunk, h = (blockIdx.x / tiles_per_chunk) % H, c = blockIdx.x / (tiles_per_chunk * H);
-  const int tok0 = tix * 128;
-  for (int i = threadIdx.x; i < 128 * 16; i += blockDim.x) {          // 16-byte pieces: row, piece (8 per 64-column atom)
-    const int row = i >> 4, piece = i & 15;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (tok0 + row < L) v = x[(((size_t)c * L + tok0 + row) * H + h) * 16 + piece];
-    *reinterpret_cast<uint4*>(tile + (piece >> 3) * 16384 + sw128_offset(row, piece & 7)) = v;
-  }
-  __syncthreads();
-  rope_rows_warp(tile, (threadIdx.x >> 5) * 16, threadIdx.x & 31, tab4, tab,
-                 [=](int row) { return tok0 + row < L ? tok0 + row : -1; });
-  __syncthreads();
-  for (int i = threadIdx.x; i < 128 * 16; i += blockDim.x) {
-    const int row = i >> 4, piece = i & 15;
-    if (tok0 + row < L)
-      y[(((size_t)c * L + tok0 + row) * H + h) * 16 + piece] =
-          *reinterpret_cast<const uint4*>(tile + (piece >> 3) * 16384 + sw128_offset(row, piece & 7));
-  }
-}
-
-void launch_rope_tiles(const void* x, void* y, const float4* tab4, const double2* tab, int C, int L, int H, cudaStream_t st) {
-  const int tiles = (L + 127) / 128;
-  rope_tiles_kernel<<<C * H * tiles, 256, 0, st>>>((const uint4*)x, (uint4*)y, tab4, tab, L, H, tiles);
+  // enough blocks in flight to cover the memory latency: split the chunks over gridDim.y when L alone is short
+  int ny = C < 64 ? C : 64;
+  dim3 grid((unsigned)((n + 255) / 256), (unsigned)ny);
+  note_launch();
+  rope_rows_kernel<<<grid, 256, 0, st>>>((const uint16_t*)x, x_stride[0], x_stride[1], x_stride[2], (uint16_t*)y, tab_hi,
+                                         tab_lo, tab, C, L, H, d);
 }
 
 }  // namespace pc

@@ -22,6 +22,7 @@ __global__ void chunk_score_kernel(const float* __restrict__ win_lse, int n_per_
 }
 
 void launch_chunk_score(const float* win_lse, int C, int n_per_chunk, float* score, cudaStream_t st) {
+  note_launch();
   chunk_score_kernel<<<C, 256, 0, st>>>(win_lse, n_per_chunk, score);
 }
 
@@ -51,6 +52,7 @@ __global__ void select_chunks_kernel(const float* __restrict__ score, int C, int
 }
 
 void launch_select_chunks(const float* score, int C, int m, int lower_is_better, int* kept, cudaStream_t st) {
+  note_launch();
   select_chunks_kernel<<<1, 1024, 0, st>>>(score, C, m, lower_is_better, kept);
 }
 
@@ -318,6 +320,7 @@ cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m,
   const int grid = m * Hkv;
 #define PC_SELECT(C, S)                                                                                               \
   do {                                                                                                                \
+    note_launch();                                                                                                    \
     if (threads <= 256)                                                                                               \
       select_tokens_kernel<C, S, true><<<grid, threads, S ? stage_bytes : 0, st>>>(win_score, kept, Hkv, L, n_cand, k, \
                                                                                     idx, cal);                        \
@@ -380,6 +383,7 @@ cudaError_t launch_gather_kv(const void* k_src, const void* v_src, const long lo
 #define PC_GATHER(D, S)                                                                                              \
   gather_kv_kernel<D, S><<<blocks, 256, 0, st>>>((const uint4*)k_src, (const uint4*)v_src, sc, stok, sh, kept, idx, m, \
                                                  Hkv, k, (uint4*)k_out, (uint4*)v_out, pos_out)
+  note_launch();
   if (d == 128) {
     if (by_slot) PC_GATHER(128, true); else PC_GATHER(128, false);
   } else {

@@ -45,11 +45,13 @@ def test_status_strings_and_version(lib):
 
 def test_workspace_queries_are_host_only(lib):
     from paper_2502_14317_b200 import binding
-    # cfg1: 256 B counter + fp64 cos/sin table L * d/2 * 16 B + its fp32 head+tail copy L * d/2 * 16 B
-    assert binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128) == 256 + 8192 * 64 * 16 + 8192 * 64 * 16
-    assert binding.chunk_prefill_attn_workspace_bytes(4, 256, 16, 4, 2, 64) == 256 + 256 * 32 * 16 + 256 * 32 * 16
+    # cfg1: 256 B counter + fp64 cos/sin table L * d/2 * 16 B + its fp32 head and tail copies 2 * L * d/2 * 8 B
+    # + the rotated queries C * L * Hq * d * 2 B
+    tables = lambda L, d: 256 + L * (d // 2) * 16 + L * (d // 2) * 16
+    assert binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128) == tables(8192, 128) + 16 * 8192 * 32 * 128 * 2
+    assert binding.chunk_prefill_attn_workspace_bytes(4, 256, 16, 4, 2, 64) == tables(256, 64) + 4 * 256 * 4 * 64 * 2
     with_krot = binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128, k_rot_in_workspace=True)
-    assert with_krot == 256 + 8192 * 64 * 16 + 8192 * 64 * 16 + 16 * 8192 * 8 * 128 * 2
+    assert with_krot == tables(8192, 128) + 16 * 8192 * 32 * 128 * 2 + 16 * 8192 * 8 * 128 * 2
     # unsupported shapes give 0
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 24, 4, 2, 64) == 0       # window not a power of two
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 2, 96) == 0       # head size
