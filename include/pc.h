@@ -13,8 +13,9 @@
  *     otherwise; d is the contiguous dimension; strides are in elements and must be
  *     multiples of 8.  Descriptor structs and stride arrays are HOST memory.
  *   - The caller owns every buffer.  The library allocates no device memory and keeps
- *     no state between calls; scratch comes from the caller's workspace, sized by the
- *     matching *_workspace_bytes query (host function, no GPU work).
+ *     no state between calls (pc_parallel_attn_static, below, is the one exception: its
+ *     scratch is an array inside the library image); scratch comes from the caller's
+ *     workspace, sized by the matching *_workspace_bytes query (host function, no GPU work).
  *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*, NULL = the
  *     default stream) and return without synchronising.  Index outputs of one call
  *     are device inputs of the next, so the five calls chain on one stream with no
@@ -22,11 +23,12 @@
  *   - Return value: PC_OK or a negative pc_status.  Argument errors are found on the
  *     host before anything is launched; nothing is written in that case.
  *   - `status_word` (device int32, may be NULL) is left untouched on success; a kernel
- *     whose bounded wait on a copy or tensor-core barrier ran out stores a non-zero
- *     code there and the results of that call are undefined.  The caller clears it and
+ *     whose bounded wait on a copy or tensor-core barrier ran out stores a positive code
+ *     naming that wait there (the condition PC_ERR_TIMEOUT stands for) and the results of
+ *     that call are undefined.  The caller clears it and
  *     reads it after synchronising.  No kernel spins without a limit.
- *   - Supported: d in {64, 128}; Hq % Hkv == 0; w a power of two in [8, 128]; w < L;
- *     G * w <= 1024 (256 window rows are handled per pass, larger groups take several).
+ *   - Supported: d in {64, 128}; Hq % Hkv == 0; any window 1 <= w < L with w <= 128;
+ *     G * w <= 1024 (the window rows of all G heads of a kv-head are swept in passes of up to 256 rows).
  */
 #ifndef PC_H_
 #define PC_H_
@@ -78,11 +80,22 @@ PC_API uint64_t pc_launch_count(void);
  * against the final log-sum-exp); it is not a separate launch.
  *
  * q [C,L,Hq,d], k, v [C,L,Hkv,d]: inputs before RoPE, addressed through the element
- * strides (chunk, token, head) in the descriptor.
+ * strides (chunk, token, head) in the descriptor.  Queries and keys are rotated by a pass
+ * of their own ahead of the attention kernel (the rotated queries live in the workspace).
+ * chunk_len [C] int32 (device; NULL: every chunk holds L tokens): tokens of chunk c, window
+ * included - the paper cuts the input into chunks of AT MOST the trained length.  The
+ * window of a shorter chunk directly follows its context (positions len-w .. len-1); keys
+ * at or behind len are masked; o, lse and win_score read as zero at positions >= len.
+ * Values outside (w, L] are clamped into that range.  The rows of k and v behind len must
+ * hold finite numbers (they meet zero probabilities).  pc_select_tokens then ranks such a
+ * chunk with n_cand = len - w (a call of its own for that chunk).
  * o [C,L,Hq,d] (strides o_stride), k_rot [C,L,Hkv,d] contiguous (rotated keys, what the
  * gather later copies; may be NULL, then it lives in the workspace), lse [C,Hq,L] fp32
  * natural-log log-sum-exp of every row (may be NULL), win_score [C,Hkv,L] fp32,
- * win_lse [C,Hq,w] fp32 (rows L-w..L-1).
+ * win_lse [C,Hq,w] fp32 (rows len-w..len-1 of each chunk).
+ * Workspace: pc_chunk_prefill_attn_workspace_bytes(desc) - cos/sin tables and the rotated
+ * queries (C*L*Hq*d bf16) - plus, if k_rot is NULL, C*L*Hkv*d*2 bytes rounded up to a
+ * multiple of 256 for the rotated keys.
  */
 typedef struct {
   int32_t C, L, w, Hq, Hkv, d;
@@ -91,11 +104,29 @@ typedef struct {
   int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];   /* chunk, token, head; 0,0,0 -> contiguous */
 } pc_prefill_desc;
 
-PC_API size_t pc_chunk_prefill_attn_workspace_bytes(const pc_prefill_desc* desc, int32_t k_rot_in_workspace);
+PC_API size_t pc_chunk_prefill_attn_workspace_bytes(const pc_prefill_desc* desc);
 
 PC_API int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const void* k, const void* v,
-                              void* o, void* k_rot, float* lse, float* win_score, float* win_lse,
-                              int32_t* status_word, void* workspace, size_t workspace_bytes, void* stream);
+                              const int32_t* chunk_len, void* o, void* k_rot, float* lse, float* win_score,
+                              float* win_lse, int32_t* status_word, void* workspace, size_t workspace_bytes,
+                              void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Test hook for the bounded device-side waits (no counterpart in the paper).
+ * Every wait of a kernel on a copy or tensor-core barrier gives up after a limit, stores a
+ * positive code naming the wait in the call's status_word, lets the kernel drain what is in
+ * flight and return; the host then treats the call's results as undefined (PC_ERR_TIMEOUT).
+ *   wait_limit_cycles      limit for all later launches of this process (0: the default of
+ *                          about 2e9 cycles, a second);
+ *   skip_final_publication non-zero: the single-CTA chunk-prefill kernel (head size 64, or an
+ *                          odd number of q-heads per kv-head) leaves out ONE signal that carries
+ *                          no data - the "no more work" message to its consumer warps after the
+ *                          last work item, when nothing is in flight any more - so that their
+ *                          wait runs out.  Outputs of such a call are complete; its status_word
+ *                          is non-zero.  Zero switches the hook off again.
+ * Host-side settings, read at every launch.
+ */
+PC_API int32_t pc_debug_bounded_wait_test(int64_t wait_limit_cycles, int32_t skip_final_publication);
 
 /* ------------------------------------------------------------------------------------
  * RoPE with position reuse on its own.  Paper: Sec. 3.1 "Parallel attention" (the position
@@ -165,13 +196,13 @@ PC_API int32_t pc_select_tokens_calibrated(const float* win_score, const int32_t
  * Compressed cache.  Paper: Eq. 7 (K[R], V[R]) and Eq. 9 (concatenation over chunks).
  *     k_out[hkv, r*k + t, :] = k_src[kept[r], idx[r,hkv,t], hkv, :]     (same for v)
  *     pos_out[hkv, r*k + t]  = idx[r,hkv,t]
- * k_src (rotated keys) and v_src are [C,L,Hkv,d] addressed by kv_stride (chunk, token,
- * head; host array; NULL -> contiguous); outputs are contiguous [Hkv, m*k, d] and
+ * k_src (rotated keys) and v_src are [C,L,Hkv,d] addressed by kv_stride (element strides of
+ * chunk, token, head; host array of 3; [L*Hkv*d, Hkv*d, d] for contiguous tensors); outputs are contiguous [Hkv, m*k, d] and
  * [Hkv, m*k] int32 (pos_out may be NULL).  Entries with idx < 0 give zero rows and
  * position -1.  Pure bit copy.
  */
-PC_API int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t* kv_stride, int32_t L,
-                     const int32_t* kept, const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d,
+PC_API int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t* kv_stride, const int32_t* kept,
+                     const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d,
                      void* k_out, void* v_out, int32_t* pos_out, void* stream);
 
 /* ------------------------------------------------------------------------------------
@@ -211,7 +242,7 @@ PC_API int32_t pc_queue_init(int32_t m, float* q_score, int32_t* q_chunk, void* 
 PC_API int32_t pc_queue_update(const float* chunk_score, int32_t Cb, int32_t chunk_id0, int32_t lower_is_better,
                         int32_t m, float* q_score, int32_t* q_chunk, int32_t* slot_src, void* stream);
 
-PC_API int32_t pc_queue_gather(const void* k_src, const void* v_src, const int64_t* kv_stride, int32_t L,
+PC_API int32_t pc_queue_gather(const void* k_src, const void* v_src, const int64_t* kv_stride,
                         const int32_t* slot_src, const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d,
                         void* q_k, void* q_v, int32_t* q_pos, void* stream);
 

@@ -6,7 +6,7 @@ There is no CPU fallback: importing :mod:`paper_2502_14317_b200.binding` raises 
 library is missing.
 """
 from .binding import (  # noqa: F401
-    PcError, lib_path, load_library, version, status_string,
+    PcError, lib_path, load_library, version, status_string, launch_count,
     chunk_prefill_attn, chunk_prefill_attn_workspace_bytes, chunk_score_from_lse, rope_position_reuse,
     select_chunks, select_tokens, select_tokens_calibrated, gather_kv, parallel_attn, parallel_attn_workspace_bytes,
     parallel_attn_static, parallel_attn_static_scratch_bytes, hot_path, hot_path_from_host,

@@ -45,13 +45,17 @@ def load_library():
     lib.pc_status_string.argtypes = [c_int32]
     lib.pc_version.restype = c_int32
     lib.pc_chunk_prefill_attn_workspace_bytes.restype = c_size_t
-    lib.pc_chunk_prefill_attn_workspace_bytes.argtypes = [POINTER(_PrefillDesc), c_int32]
+    lib.pc_chunk_prefill_attn_workspace_bytes.argtypes = [POINTER(_PrefillDesc)]
     lib.pc_chunk_prefill_attn.restype = c_int32
-    lib.pc_chunk_prefill_attn.argtypes = [POINTER(_PrefillDesc)] + [c_void_p] * 10 + [c_size_t, c_void_p]
+    lib.pc_chunk_prefill_attn.argtypes = [POINTER(_PrefillDesc)] + [c_void_p] * 11 + [c_size_t, c_void_p]
     lib.pc_rope_position_reuse_workspace_bytes.restype = c_size_t
     lib.pc_rope_position_reuse_workspace_bytes.argtypes = [c_int32, c_int32]
     lib.pc_rope_position_reuse.restype = c_int32
     lib.pc_rope_position_reuse.argtypes = [c_void_p] + [c_int32] * 4 + [c_float, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.pc_debug_bounded_wait_test.restype = c_int32
+    lib.pc_debug_bounded_wait_test.argtypes = [c_int64, c_int32]
+    lib.pc_launch_count.restype = ctypes.c_uint64
+    lib.pc_launch_count.argtypes = []
     lib.pc_chunk_score_from_lse.restype = c_int32
     lib.pc_chunk_score_from_lse.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
     lib.pc_select_chunks.restype = c_int32
@@ -61,14 +65,14 @@ def load_library():
     lib.pc_select_tokens_calibrated.restype = c_int32
     lib.pc_select_tokens_calibrated.argtypes = [c_void_p, c_void_p] + [c_int32] * 8 + [c_float] * 3 + [c_void_p, c_void_p]
     lib.pc_gather_kv.restype = c_int32
-    lib.pc_gather_kv.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_int32, c_void_p, c_void_p] + [c_int32] * 4 + \
+    lib.pc_gather_kv.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_void_p, c_void_p] + [c_int32] * 4 + \
                                 [c_void_p, c_void_p, c_void_p, c_void_p]
     lib.pc_queue_init.restype = c_int32
     lib.pc_queue_init.argtypes = [c_int32, c_void_p, c_void_p, c_void_p]
     lib.pc_queue_update.restype = c_int32
     lib.pc_queue_update.argtypes = [c_void_p] + [c_int32] * 4 + [c_void_p] * 4
     lib.pc_queue_gather.restype = c_int32
-    lib.pc_queue_gather.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_int32, c_void_p, c_void_p] + [c_int32] * 4 + \
+    lib.pc_queue_gather.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_void_p, c_void_p] + [c_int32] * 4 + \
         [c_void_p] * 4
     lib.pc_queue_emit.restype = c_int32
     lib.pc_queue_emit.argtypes = [c_void_p] + [c_int32] * 4 + [c_void_p] * 9
@@ -87,6 +91,11 @@ def load_library():
 
 def version() -> int:
     return int(load_library().pc_version())
+
+
+def launch_count() -> int:
+    """pc_launch_count: kernels launched by the library in this process so far."""
+    return int(load_library().pc_launch_count())
 
 
 def status_string(code: int) -> str:
@@ -125,12 +134,16 @@ def _make_desc(q, k, v, o, w, rope_theta, softmax_scale):
 
 def chunk_prefill_attn_workspace_bytes(C, L, w, Hq, Hkv, d, k_rot_in_workspace=False) -> int:
     desc = _PrefillDesc(C, L, w, Hq, Hkv, d, 10000.0, 0.0)
-    return int(load_library().pc_chunk_prefill_attn_workspace_bytes(ctypes.byref(desc), int(k_rot_in_workspace)))
+    need = int(load_library().pc_chunk_prefill_attn_workspace_bytes(ctypes.byref(desc)))
+    if need and k_rot_in_workspace:                           # rotated keys in the workspace (k_rot = NULL in the call)
+        need += (C * L * Hkv * d * 2 + 255) // 256 * 256
+    return need
 
 
 def chunk_prefill_attn(q, k, v, *, w, rope_theta, softmax_scale=0.0, want_lse=False, out=None, k_rot=None,
-                       win_score=None, win_lse=None, lse=None, status=None, workspace=None):
-    """pc_chunk_prefill_attn: q [C,L,Hq,d], k/v [C,L,Hkv,d] bf16 (pre-RoPE).
+                       win_score=None, win_lse=None, lse=None, status=None, workspace=None, chunk_len=None):
+    """pc_chunk_prefill_attn: q [C,L,Hq,d], k/v [C,L,Hkv,d] bf16 (pre-RoPE); chunk_len: int32 [C] device tensor
+    (tokens per chunk, window included) or None for full chunks.
 
     Returns dict(o, k_rot, win_score, win_lse, lse, status, workspace).
     """
@@ -151,12 +164,14 @@ def chunk_prefill_attn(q, k, v, *, w, rope_theta, softmax_scale=0.0, want_lse=Fa
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
     desc = _make_desc(q, k, v, o, w, rope_theta, softmax_scale)
-    need = int(lib.pc_chunk_prefill_attn_workspace_bytes(ctypes.byref(desc), 0))
+    need = int(lib.pc_chunk_prefill_attn_workspace_bytes(ctypes.byref(desc)))
     if workspace is None or workspace.numel() < need:          # need == 0: a bad descriptor, which the call below names
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
-    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(k_rot), _ptr(lse),
-                                   _ptr(win_score), _ptr(win_lse), _ptr(status), _ptr(workspace), workspace.numel(),
-                                   _stream())
+    if chunk_len is not None and (chunk_len.dtype != torch.int32 or chunk_len.numel() != C or not chunk_len.is_cuda):
+        raise PcError("chunk_len must be an int32 CUDA tensor with one entry per chunk")
+    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(chunk_len), _ptr(o), _ptr(k_rot),
+                                   _ptr(lse), _ptr(win_score), _ptr(win_lse), _ptr(status), _ptr(workspace),
+                                   workspace.numel(), _stream())
     _check(rc, "pc_chunk_prefill_attn")
     return {"o": o, "k_rot": k_rot, "win_score": win_score, "win_lse": win_lse, "lse": lse, "status": status,
             "workspace": workspace}
@@ -239,7 +254,7 @@ def gather_kv(k_src, v_src, kept, idx, k_out=None, v_out=None, pos_out=None, wan
     if pos_out is None and want_pos:
         pos_out = torch.empty((Hkv, m * k), dtype=torch.int32, device=dev)
     strides = (c_int64 * 3)(k_src.stride(0), k_src.stride(1), k_src.stride(2))
-    _check(lib.pc_gather_kv(_ptr(k_src), _ptr(v_src), strides, L, _ptr(kept), _ptr(idx), m, Hkv, k, d, _ptr(k_out),
+    _check(lib.pc_gather_kv(_ptr(k_src), _ptr(v_src), strides, _ptr(kept), _ptr(idx), m, Hkv, k, d, _ptr(k_out),
                             _ptr(v_out), _ptr(pos_out), _stream()), "pc_gather_kv")
     return k_out, v_out, pos_out
 
@@ -286,7 +301,7 @@ def queue_gather(state, k_src, v_src, idx):
     if k_src.stride() != v_src.stride() or k_src.stride(3) != 1:
         raise PcError("k_src and v_src must share strides with a contiguous head dimension")
     strides = (c_int64 * 3)(k_src.stride(0), k_src.stride(1), k_src.stride(2))
-    _check(lib.pc_queue_gather(_ptr(k_src), _ptr(v_src), strides, L, _ptr(state["slot_src"]), _ptr(idx), state["m"], Hkv,
+    _check(lib.pc_queue_gather(_ptr(k_src), _ptr(v_src), strides, _ptr(state["slot_src"]), _ptr(idx), state["m"], Hkv,
                                state["k"], d, _ptr(state["q_k"]), _ptr(state["q_v"]), _ptr(state["q_pos"]), _stream()),
            "pc_queue_gather")
 

@@ -12,6 +12,8 @@
 namespace pc {
 static std::atomic<unsigned long long> g_launches{0};
 void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+static std::atomic<int> g_wait_kcycles{1 << 21};            // limit of the device-side waits, units of 1024 cycles (~1 s)
+static std::atomic<int> g_skip_final_publication{0};        // test hook, see pc_debug_bounded_wait_test
 }  // namespace pc
 
 namespace {
@@ -69,7 +71,7 @@ int32_t check_prefill_desc(const pc_prefill_desc* d) {
   if (d->C < 1 || d->L < 2 || d->w < 1 || d->w >= d->L || d->Hq < 1 || d->Hkv < 1 || d->Hq % d->Hkv != 0) return PC_ERR_INVALID_ARG;
   if (!(d->rope_theta > 0.0f) || d->softmax_scale < 0.0f) return PC_ERR_INVALID_ARG;
   if (d->d != 64 && d->d != 128) return PC_ERR_UNSUPPORTED;
-  if (!pow2_between(d->w, 8, 128)) return PC_ERR_UNSUPPORTED;
+  if (d->w > 128) return PC_ERR_UNSUPPORTED;
   if ((int64_t)(d->Hq / d->Hkv) * d->w > 1024) return PC_ERR_UNSUPPORTED;
   if ((int64_t)d->C * d->Hkv > (1 << 24) || d->L > (1 << 24)) return PC_ERR_UNSUPPORTED;
   return PC_OK;
@@ -96,15 +98,24 @@ int32_t pc_version(void) { return 1001; }
 
 uint64_t pc_launch_count(void) { return pc::g_launches.load(std::memory_order_relaxed); }
 
-// ------------------------------------------------------------------------------------ prefill
-size_t pc_chunk_prefill_attn_workspace_bytes(const pc_prefill_desc* desc, int32_t k_rot_in_workspace) {
-  if (check_prefill_desc(desc) != PC_OK) return 0;
-  return prefill_layout(desc, k_rot_in_workspace != 0).total;
+int32_t pc_debug_bounded_wait_test(int64_t wait_limit_cycles, int32_t skip_final_publication) {
+  if (wait_limit_cycles < 0 || wait_limit_cycles > (int64_t)2000000000 * 1024) return PC_ERR_INVALID_ARG;
+  const int64_t kc = wait_limit_cycles == 0 ? (1 << 21) : (wait_limit_cycles + 1023) / 1024;
+  pc::g_wait_kcycles.store((int)(kc < 1 ? 1 : kc));
+  pc::g_skip_final_publication.store(skip_final_publication != 0 ? 1 : 0);
+  return PC_OK;
 }
 
-int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const void* k, const void* v, void* o,
-                              void* k_rot, float* lse, float* win_score, float* win_lse, int32_t* status_word,
-                              void* workspace, size_t workspace_bytes, void* stream) {
+// ------------------------------------------------------------------------------------ prefill
+size_t pc_chunk_prefill_attn_workspace_bytes(const pc_prefill_desc* desc) {
+  if (check_prefill_desc(desc) != PC_OK) return 0;
+  return prefill_layout(desc, false).total;
+}
+
+int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const void* k, const void* v,
+                              const int32_t* chunk_len, void* o, void* k_rot, float* lse, float* win_score,
+                              float* win_lse, int32_t* status_word, void* workspace, size_t workspace_bytes,
+                              void* stream) {
   int32_t rc = check_prefill_desc(desc);
   if (rc != PC_OK) return rc;
   if (!q || !k || !v || !o || !win_score || !win_lse) return PC_ERR_INVALID_ARG;
@@ -141,7 +152,7 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
   const uint64_t o_str[3] = {(uint64_t)os[2], (uint64_t)os[1], (uint64_t)os[0]};
   const uint64_t kr_str[3] = {(uint64_t)d, (uint64_t)desc->Hkv * d, (uint64_t)desc->L * desc->Hkv * d};
   const uint32_t box_tile[4] = {64, 1, 128, 1};
-  const uint32_t box_win[4] = {64, 1, (uint32_t)desc->w, 1};
+  const uint32_t box_win[4] = {64, 1, (uint32_t)((desc->w + 7) & ~7), 1};   // window rows of a head in the score sweep, padded to 8
   const uint32_t box_half[4] = {64, 1, 64, 1};
   if (!pc::make_tmap_bf16_4d(&maps[0], qrot, q_dims, q_str, box_tile) ||
       !pc::make_tmap_bf16_4d(&maps[1], krot, kv_dims, kr_str, box_tile) ||
@@ -154,16 +165,22 @@ int32_t pc_chunk_prefill_attn(const pc_prefill_desc* desc, const void* q, const 
   if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return PC_ERR_CUDA;
   pc::launch_rope_table(table, table_hi, table_lo, desc->L, d, (double)desc->rope_theta, 0, st);
   // queries and keys are rotated once, ahead of the attention kernel (positions 0 .. L-1 in every chunk)
-  const long long ks_ll[3] = {ks[0], ks[1], ks[2]}, qs_ll[3] = {qs[0], qs[1], qs[2]};
+  const long long ks_ll[3] = {ks[0], ks[1], ks[2]}, qs_ll[3] = {qs[0], qs[1], qs[2]}, os_ll[3] = {os[0], os[1], os[2]};
   pc::launch_rope_rows(k, ks_ll, krot, table, table_hi, table_lo, desc->C, desc->L, desc->Hkv, d, st);
   pc::launch_rope_rows(q, qs_ll, qrot, table, table_hi, table_lo, desc->C, desc->L, desc->Hq, d, st);
 
+  if (chunk_len != nullptr)   // rows and scores behind the end of a shorter chunk read as zero: the kernels below skip them
+    pc::launch_zero_chunk_tails(chunk_len, desc->C, desc->L, desc->w, desc->Hq, desc->Hkv, d, o, os_ll, lse, win_score, st);
+
   pc::PrefillParams prm;
+  prm.chunk_len = chunk_len;
   prm.C = desc->C; prm.L = desc->L; prm.w = desc->w; prm.Hq = desc->Hq; prm.Hkv = desc->Hkv;
   const double scale = desc->softmax_scale > 0.0f ? (double)desc->softmax_scale : 1.0 / std::sqrt((double)d);
   prm.scale_log2 = (float)(scale * 1.4426950408889634);
   prm.lse = lse; prm.win_lse = win_lse; prm.win_score = win_score;
   prm.status = status_word; prm.counter = counter;
+  prm.wait_kcycles = pc::g_wait_kcycles.load();
+  prm.skip_final_publication = pc::g_skip_final_publication.load();
   // head size 128 with an even number of q-heads per kv-head runs on CTA pairs (cta_group::2: the two CTAs take
   // the same query tile of two heads that share K/V); head size 64 and odd group sizes (multi-head attention:
   // one q-head per kv-head) run on single CTAs with two query blocks each
@@ -249,16 +266,14 @@ int32_t pc_select_tokens_calibrated(const float* win_score, const int32_t* kept,
 }
 
 // ------------------------------------------------------------------------------------ gather
-int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t* kv_stride, int32_t L, const int32_t* kept,
+int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t* kv_stride, const int32_t* kept,
                      const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d, void* k_out, void* v_out,
                      int32_t* pos_out, void* stream) {
-  if (!k_src || !v_src || !kept || !idx || !k_out || !v_out) return PC_ERR_INVALID_ARG;
-  if (m < 1 || Hkv < 1 || k < 1 || L < 1) return PC_ERR_INVALID_ARG;
+  if (!k_src || !v_src || !kv_stride || !kept || !idx || !k_out || !v_out) return PC_ERR_INVALID_ARG;
+  if (m < 1 || Hkv < 1 || k < 1) return PC_ERR_INVALID_ARG;
   if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
   if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(k_out) || !aligned16(v_out)) return PC_ERR_INVALID_ARG;
-  long long s[3];
-  if (kv_stride) { s[0] = kv_stride[0]; s[1] = kv_stride[1]; s[2] = kv_stride[2]; }
-  else { s[0] = (long long)L * Hkv * d; s[1] = (long long)Hkv * d; s[2] = d; }
+  const long long s[3] = {kv_stride[0], kv_stride[1], kv_stride[2]};
   if (s[0] <= 0 || s[1] <= 0 || s[2] < d || s[0] % 8 || s[1] % 8 || s[2] % 8) return PC_ERR_INVALID_ARG;
   const DeviceInfo& dev = device_info();
   if (dev.ok != 1) return PC_ERR_UNSUPPORTED;
@@ -288,16 +303,14 @@ int32_t pc_queue_update(const float* chunk_score, int32_t Cb, int32_t chunk_id0,
   return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
 }
 
-int32_t pc_queue_gather(const void* k_src, const void* v_src, const int64_t* kv_stride, int32_t L,
+int32_t pc_queue_gather(const void* k_src, const void* v_src, const int64_t* kv_stride,
                         const int32_t* slot_src, const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d,
                         void* q_k, void* q_v, int32_t* q_pos, void* stream) {
-  if (!k_src || !v_src || !slot_src || !idx || !q_k || !q_v || !q_pos) return PC_ERR_INVALID_ARG;
-  if (m < 1 || Hkv < 1 || k < 1 || L < 1) return PC_ERR_INVALID_ARG;
+  if (!k_src || !v_src || !kv_stride || !slot_src || !idx || !q_k || !q_v || !q_pos) return PC_ERR_INVALID_ARG;
+  if (m < 1 || Hkv < 1 || k < 1) return PC_ERR_INVALID_ARG;
   if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
   if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(q_k) || !aligned16(q_v)) return PC_ERR_INVALID_ARG;
-  long long s[3];
-  if (kv_stride) { s[0] = kv_stride[0]; s[1] = kv_stride[1]; s[2] = kv_stride[2]; }
-  else { s[0] = (long long)L * Hkv * d; s[1] = (long long)Hkv * d; s[2] = d; }
+  const long long s[3] = {kv_stride[0], kv_stride[1], kv_stride[2]};
   if (s[0] <= 0 || s[1] <= 0 || s[2] < d || s[0] % 8 || s[1] % 8 || s[2] % 8) return PC_ERR_INVALID_ARG;
   const DeviceInfo& dev = device_info();
   if (dev.ok != 1) return PC_ERR_UNSUPPORTED;
@@ -438,6 +451,7 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   prm.lse_out = lse_out;
   prm.status = status_word;
   prm.counter = counter;
+  prm.wait_kcycles = pc::g_wait_kcycles.load();
   const long long n_items = (long long)B * Hkv * plan.n_rg * plan.n_split;
   const int grid = (int)(n_items < dev.sm_count ? n_items : dev.sm_count);
   if (pc::launch_parallel_attn(maps, prm, d, grid, st) != cudaSuccess) return PC_ERR_CUDA;

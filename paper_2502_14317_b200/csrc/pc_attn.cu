@@ -50,9 +50,11 @@ struct __align__(16) Misc {
   uint64_t item_full[2], item_empty[2];
   uint64_t t_full[2], t_free[2];
   uint64_t turn[2];                        // issue token passed between the two tcgen05 issuers
+  uint64_t mma_done;                       // every tensor-core operation of both issuers has completed (teardown)
   int item_slot[2];
   uint32_t tmem_base;
-  int abort_flag;
+  int abort_flag;                          // these two words stay adjacent: bounded waits read the limit through the
+  int wait_kcycles;                        // flag's address
   float lse2[1024];                        // window-row log-sum-exp (log2 domain), G * w <= 1024
   float xch[2][TILE];
 };
@@ -73,9 +75,23 @@ struct SubItem {
 };
 
 // ------------------------------------------------------------------ item decoding (prefill)
+// With per-chunk lengths the query tiles of a shorter chunk are numbered from the END: slot v of the static
+// decomposition (v = T - 1 is the last tile of a full-length chunk) is tile v - (T - T_c) of a chunk with T_c
+// tiles; slots below T - T_c are empty.  The window then always sits in the last two slots, which the tail item
+// of the group owns together with the score sweep.
 struct Sched {
   int T, t_w, ntt, G, P, hp_mode, ipg, n_lp;
+  int wp, hb, Gs, n_pass;                    // score sweep: operand rows per head (w rounded up to 8), heads per 128-row
+                                             // block, heads per pass, passes
 };
+
+// length of chunk c in tokens (window included), clamped to (w, L]
+__device__ __forceinline__ int chunk_length(const PrefillParams& p, int c) {
+  if (p.chunk_len == nullptr) return p.L;
+  int len = __ldg(p.chunk_len + c);
+  len = len > p.L ? p.L : len;
+  return len <= p.w ? p.w + 1 : len;
+}
 
 __device__ __forceinline__ Sched make_sched(const PrefillParams& p) {
   Sched s;
@@ -83,9 +99,16 @@ __device__ __forceinline__ Sched make_sched(const PrefillParams& p) {
   s.G = p.Hq / p.Hkv;
   s.hp_mode = (s.G % 2 == 0);
   s.P = s.G / 2;
+  s.wp = (p.w + 7) & ~7;
+  s.hb = TILE / s.wp;
+  s.Gs = 2 * s.hb < s.G ? 2 * s.hb : s.G;
+  s.n_pass = (s.G + s.Gs - 1) / s.Gs;
   if (s.hp_mode) {
-    s.t_w = (p.L - p.w) / TILE;              // first tile holding a window row
-    s.ntt = s.T - s.t_w;                     // 1 or 2 tail tiles
+    // tail slots: the tiles that can hold window rows (two with per-chunk lengths: the window of some chunk may
+    // straddle two tiles even where that of a full-length chunk does not)
+    s.ntt = (p.chunk_len != nullptr) ? (p.w > 1 ? 2 : 1) : s.T - (p.L - p.w) / TILE;
+    if (s.ntt > s.T) s.ntt = s.T;
+    s.t_w = s.T - s.ntt;
     s.n_lp = 0;
     s.ipg = 1 + s.t_w * s.P;
   } else {
@@ -97,13 +120,21 @@ __device__ __forceinline__ Sched make_sched(const PrefillParams& p) {
   return s;
 }
 
+// score sweep: q-heads whose window rows sit in block b (0 / 1) of pass u
+__device__ __forceinline__ int sweep_heads(const Sched& s, int u, int b) {
+  const int heads = (s.G - u * s.Gs) < s.Gs ? (s.G - u * s.Gs) : s.Gs;
+  const int first = heads < s.hb ? heads : s.hb;
+  return b ? heads - first : first;
+}
+
 // number of sub-items of item `within` (0 = tail item of the group)
 __device__ __forceinline__ int n_subitems(const Sched& s, int within) {
   if (within != 0) return 1;
   return s.hp_mode ? s.P * s.ntt : s.G;
 }
 
-__device__ __forceinline__ SubItem decode_sub(const Sched& s, int hkv, int within, int sub) {
+// len: length of the sub-item's chunk.  Returns hA < 0 for an empty sub-item (every role skips it).
+__device__ __forceinline__ SubItem decode_sub(const Sched& s, int hkv, int within, int sub, int len) {
   SubItem it;
   const int h0 = hkv * s.G;
   if (s.hp_mode) {
@@ -117,6 +148,16 @@ __device__ __forceinline__ SubItem decode_sub(const Sched& s, int hkv, int withi
     else { const int x = within - 1; g = x % s.G; hi = s.t_w - 1 - 2 * (x / s.G); }
     if (hi >= 1) { it.hA = h0 + g; it.tA = hi - 1; it.hB = h0 + g; it.tB = hi; }
     else { it.hA = h0 + g; it.tA = hi; it.hB = -1; it.tB = 0; }
+  }
+  const int shift = s.T - (len + TILE - 1) / TILE;          // empty slots of a shorter chunk
+  if (shift > 0) {
+    it.tA -= shift;
+    it.tB -= shift;
+    if (it.hB >= 0 && it.tB < 0) it.hB = -1;
+    if (it.tA < 0) {
+      if (it.hB >= 0 && s.hp_mode == 0) { it.tA = it.tB; it.hB = -1; it.tB = 0; }   // only the upper tile of the pair exists
+      else { it.hA = -1; it.hB = -1; }
+    }
   }
   return it;
 }
@@ -280,7 +321,7 @@ struct Ctx {
   int* status;
 };
 
-__device__ __forceinline__ void init_barriers(Misc& mi) {
+__device__ __forceinline__ void init_barriers(Misc& mi, int wait_kcycles) {
 #pragma unroll
   for (int b = 0; b < 2; ++b) {
     mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 128); mbar_init(&mi.q_free[b], 1);
@@ -291,19 +332,23 @@ __device__ __forceinline__ void init_barriers(Misc& mi) {
     mbar_init(&mi.turn[b], 1);
   }
   for (int s = 0; s < NS; ++s) { mbar_init(&mi.kv_full[s], 1); mbar_init(&mi.kv_free[s], 2); }   // both issuers release a stage
+  mbar_init(&mi.mma_done, 2);
   mi.abort_flag = 0;
+  mi.wait_kcycles = wait_kcycles;
   fence_mbar_init();
 }
 
 // producer: publish the next work item (dynamic queue); returns it
-__device__ __forceinline__ int producer_next_item(const Ctx& cx, Waits& wt, int* counter, int n_items) {
+// skip_final: test hook - the "no more work" message is written but never signalled, so that the consumers' wait for
+// it runs out.  Nothing is in flight at that point: every copy has been consumed and every accumulator read out.
+__device__ __forceinline__ int producer_next_item(const Ctx& cx, Waits& wt, int* counter, int n_items, bool skip_final = false) {
   Misc& mi = *cx.mi;
   const int slot = wt.item & 1;
   mbar_wait(&mi.item_empty[slot], free_par(wt.item >> 1), cx.abort_flag, cx.status, W_ITEM);
   int item = atomicAdd(counter, 1);
   if (item >= n_items || *cx.abort_flag) item = ITEM_DONE;
   mi.item_slot[slot] = item;
-  mbar_arrive(&mi.item_full[slot]);
+  if (!(skip_final && item == ITEM_DONE)) mbar_arrive(&mi.item_full[slot]);
   ++wt.item;
   return item;
 }
@@ -311,7 +356,7 @@ __device__ __forceinline__ int producer_next_item(const Ctx& cx, Waits& wt, int*
 __device__ __forceinline__ int consumer_next_item(const Ctx& cx, Waits& wt) {
   Misc& mi = *cx.mi;
   const int slot = wt.item & 1;
-  mbar_wait(&mi.item_full[slot], full_par(wt.item >> 1), cx.abort_flag, cx.status, W_ITEM);
+  if (!mbar_wait(&mi.item_full[slot], full_par(wt.item >> 1), cx.abort_flag, cx.status, W_ITEM)) return ITEM_DONE;   // aborted: stop
   const int item = mi.item_slot[slot];
   mbar_arrive(&mi.item_empty[slot]);
   ++wt.item;
@@ -335,10 +380,10 @@ __device__ __forceinline__ void producer_ring_tile(const Ctx& cx, Waits& wt, con
 // producer: before exit, every copy it issued must have landed
 __device__ __forceinline__ void producer_drain(const Ctx& cx, const Waits& wt) {
   Misc& mi = *cx.mi;
-  for (uint32_t i = (wt.kv > NS ? wt.kv - NS : 0); i < wt.kv; ++i) mbar_wait_drain(&mi.kv_full[i % NS], full_par(i / NS));
+  for (uint32_t i = (wt.kv > NS ? wt.kv - NS : 0); i < wt.kv; ++i) mbar_wait_drain(&mi.kv_full[i % NS], full_par(i / NS), cx.abort_flag);
 #pragma unroll
   for (int b = 0; b < 2; ++b)
-    if (wt.q[b] > 0) mbar_wait_drain(&mi.q_full[b], full_par(wt.q[b] - 1));
+    if (wt.q[b] > 0) mbar_wait_drain(&mi.q_full[b], full_par(wt.q[b] - 1), cx.abort_flag);
 }
 
 // The two issuers take turns: the tensor pipe then runs the batch of one block to its end
@@ -474,10 +519,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Sched sch = make_sched(prm);
   const int n_items = prm.C * prm.Hkv * sch.ipg;
-  const int Gs = (256 / prm.w) < sch.G ? (256 / prm.w) : sch.G;      // q-heads per score pass
-  const int n_pass = (sch.G + Gs - 1) / Gs;
+  const int n_pass = sch.n_pass;
 
-  if (tid == 0) init_barriers(mi);
+  if (tid == 0) init_barriers(mi, prm.wait_kcycles);
   if (warp == WARP_MMA) tmem_alloc(&mi.tmem_base, 512);
   tc_fence_before_sync();
   __syncthreads();
@@ -491,13 +535,16 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_qw);
       while (true) {
-        const int item = producer_next_item(cx, wt, prm.counter, n_items);
+        const int item = producer_next_item(cx, wt, prm.counter, n_items, prm.skip_final_publication != 0);
         if (item == ITEM_DONE) break;
         const int group = item / sch.ipg, within = item % sch.ipg;
         const int c = group / prm.Hkv, hkv = group % prm.Hkv;
         const int nsub = n_subitems(sch, within);
+        const int len = chunk_length(prm, c);
+        const int T_c = (len + TILE - 1) / TILE;
         for (int sub = 0; sub < nsub; ++sub) {
-          const SubItem it = decode_sub(sch, hkv, within, sub);
+          const SubItem it = decode_sub(sch, hkv, within, sub, len);
+          if (it.hA < 0) continue;
 #pragma unroll
           for (int b = 0; b < 2; ++b) {
             const int h = b ? it.hB : it.hA, t = b ? it.tB : it.tA;
@@ -515,25 +562,25 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
         if (within == 0) {
-          // ---- score sweep: window queries of Gs heads per pass, then all key tiles
+          // ---- score sweep: window queries of Gs heads per pass, then all key tiles.  A head's rows in the operand
+          // are the wp tokens that end with the chunk (wp = w rounded up to 8: the first wp - w of them are not
+          // window rows and are left out of the sums; a start before token 0 reads zeros)
           for (int u = 0; u < n_pass; ++u) {
-            const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
-            const int rows_total = heads * prm.w;
 #pragma unroll
             for (int b = 0; b < 2; ++b) {
-              const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
-              if (rows_b == 0) continue;
+              const int heads_b = sweep_heads(sch, u, b);
+              if (heads_b == 0) continue;
               mbar_wait(&mi.q_free[b], free_par(wt.q[b]), cx.abort_flag, cx.status, W_QFREE);
-              mbar_arrive_expect_tx(&mi.q_full[b], rows_b * D * 2);
-              for (int r0 = 0; r0 < rows_b; r0 += prm.w) {
-                const int g = u * Gs + (b * TILE + r0) / prm.w;
+              mbar_arrive_expect_tx(&mi.q_full[b], heads_b * sch.wp * D * 2);
+              for (int ih = 0; ih < heads_b; ++ih) {
+                const int g = u * sch.Gs + b * sch.hb + ih;
                 for (int a = 0; a < C::ATOMS; ++a)
-                  tma_load_4d(cx.sQ[b] + a * 16384 + r0 * 128, &tm_qw, &mi.q_full[b], a * 64, hkv * sch.G + g,
-                              prm.L - prm.w, c);
+                  tma_load_4d(cx.sQ[b] + a * 16384 + ih * sch.wp * 128, &tm_qw, &mi.q_full[b], a * 64, hkv * sch.G + g,
+                              len - sch.wp, c);
               }
               ++wt.q[b];
             }
-            for (int j = 0; j < sch.T; ++j) producer_ring_tile<D>(cx, wt, &tm_k, hkv, j * TILE, c);
+            for (int j = 0; j < T_c; ++j) producer_ring_tile<D>(cx, wt, &tm_k, hkv, j * TILE, c);
           }
         }
       }
@@ -552,8 +599,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int group = item / sch.ipg, within = item % sch.ipg;
         const int hkv = group % prm.Hkv;
         const int nsub = n_subitems(sch, within);
+        const int len = chunk_length(prm, group / prm.Hkv);
+        const int T_c = (len + TILE - 1) / TILE;
         for (int sub = 0; sub < nsub; ++sub) {
-          const SubItem it = decode_sub(sch, hkv, within, sub);
+          const SubItem it = decode_sub(sch, hkv, within, sub, len);
+          if (it.hA < 0) continue;
           const bool has_b = (b == 0) || it.hB >= 0;
           const int nb_b = (b == 0) ? it.tA + 1 : (it.hB >= 0 ? it.tB + 1 : 0);
           const int n = (it.hB >= 0 ? it.tB : it.tA) + 1;
@@ -563,11 +613,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           // ---- score sweep: this issuer computes the columns of its own block (window rows b*128..)
           mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
           for (int u = 0; u < n_pass; ++u) {
-            const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
-            const int rows_total = heads * prm.w;
-            const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
+            const int rows_b = sweep_heads(sch, u, b) * sch.wp;
             if (rows_b > 0) { mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT); ++wt.q[b]; }
-            for (int j = 0; j < sch.T; ++j) {
+            for (int j = 0; j < T_c; ++j) {
               const int e = j & 1;
               mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
               const int st = wt.kv % NS;
@@ -587,6 +635,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
       }
+      mma_commit(&mi.mma_done);                              // teardown waits for everything this thread issued
     }
     __syncwarp();
   } else if (warp < 8) {
@@ -604,8 +653,10 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int group = item / sch.ipg, within = item % sch.ipg;
       const int c = group / prm.Hkv, hkv = group % prm.Hkv;
       const int nsub = n_subitems(sch, within);
+      const int len = chunk_length(prm, c);
+      const int T_c = (len + TILE - 1) / TILE;
       for (int sub = 0; sub < nsub; ++sub) {
-        const SubItem it = decode_sub(sch, hkv, within, sub);
+        const SubItem it = decode_sub(sch, hkv, within, sub, len);
         const int h = b ? it.hB : it.hA, t = b ? it.tB : it.tA;
         if (h < 0) continue;
         const int token = t * TILE + r;
@@ -616,6 +667,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                          [&](int j) { return (j == n - 1) ? (token - j * TILE + 1) : TILE; }, m_used, l_run);
         // ---- epilogue: normalise, stage bf16 rows in the (now idle) Q buffer, TMA store
         const float inv_l = 1.0f / l_run;
+        const bool in_chunk = token < len;                   // rows behind the end of the chunk are written as zeros
 #pragma unroll
         for (int q = 0; q < D / 32; ++q) {
           uint32_t o[32];
@@ -626,7 +678,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             uint32_t pk[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-              pk[e] = pack_bf16x2(__uint_as_float(o[g4 * 8 + 2 * e]) * inv_l, __uint_as_float(o[g4 * 8 + 2 * e + 1]) * inv_l);
+              pk[e] = in_chunk ? pack_bf16x2(__uint_as_float(o[g4 * 8 + 2 * e]) * inv_l, __uint_as_float(o[g4 * 8 + 2 * e + 1]) * inv_l) : 0u;
             const int col = q * 32 + g4 * 8;
             *reinterpret_cast<uint4*>(myQ + (col / 64) * 16384 + sw128_offset(r, (col % 64) / 8)) =
                 make_uint4(pk[0], pk[1], pk[2], pk[3]);
@@ -635,9 +687,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tc_fence_before_sync();
         mbar_arrive(&mi.acc_free[b]);
         const float lse2 = m_used + log2f(l_run);
-        if (token < prm.L) {
+        if (in_chunk) {
           if (prm.lse) prm.lse[((size_t)c * prm.Hq + h) * prm.L + token] = lse2 * 0.6931471805599453f;
-          const int wi = token - (prm.L - prm.w);
+          const int wi = token - (len - prm.w);
           if (wi >= 0) {
             prm.win_lse[((size_t)c * prm.Hq + h) * prm.w + wi] = lse2 * 0.6931471805599453f;
             if (within == 0) mi.lse2[(h - hkv * sch.G) * prm.w + wi] = lse2;
@@ -655,30 +707,31 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (within == 0) {
         // ---- score sweep: this thread owns key (j * 128 + r); columns are the window rows
         named_barrier_sync(3, 256);                           // lse2 complete and visible to both groups
+        const int w0 = len - prm.w;                           // first window token of this chunk
         for (int u = 0; u < n_pass; ++u) {
-          const int heads = (sch.G - u * Gs) < Gs ? (sch.G - u * Gs) : Gs;
-          const int rows_total = heads * prm.w;
-          const int rows_b = b ? (rows_total > TILE ? rows_total - TILE : 0) : (rows_total < TILE ? rows_total : TILE);
-          const float* lse_rows = mi.lse2 + u * Gs * prm.w + b * TILE;   // log-sum-exp of the window row on column n
-          for (int j = 0; j < sch.T; ++j) {
+          const int heads_b = sweep_heads(sch, u, b);          // heads whose rows sit in this group's columns
+          const int rows_b = heads_b * sch.wp;
+          const float* lse_rows = mi.lse2 + (u * sch.Gs + b * sch.hb) * prm.w;   // log-sum-exp of this group's first head
+          for (int j = 0; j < T_c; ++j) {
             const int e = j & 1;
             mbar_wait(&mi.t_full[e], full_par(e ? n_t1 : n_t0), cx.abort_flag, cx.status, W_TFULL);
             if (e) ++n_t1; else ++n_t0;
             tc_fence_after_sync();
             const int key = j * TILE + r;
-            const bool need_mask = (j * TILE + TILE - 1) > (prm.L - prm.w);
+            const bool need_mask = (j * TILE + TILE - 1) > w0;
             float part = 0.0f;
             const uint32_t tT = cx.tmem + e * 256 + b * 128 + lane_sel;
-            for (int c0 = 0; c0 < rows_b; c0 += 32) {
-              uint32_t sv[32];
-              tmem_ld32(tT + c0, sv);
-              tmem_wait_ld();
+            for (int ih = 0; ih < heads_b; ++ih) {             // a head has wp columns, the last w of them are window rows
+              for (int col = 0; col < sch.wp; col += 8) {
+                uint32_t sv[8];
+                tmem_ld8(tT + ih * sch.wp + col, sv);
+                tmem_wait_ld();
+                const int wi0 = col - (sch.wp - prm.w);        // window row of the first of these columns (negative: none)
 #pragma unroll
-              for (int jj = 0; jj < 32; ++jj) {
-                const int ncol = c0 + jj;
-                if (ncol < rows_b) {
-                  float pv = fast_exp2(fmaf(__uint_as_float(sv[jj]), scale_log2, -lse_rows[ncol]));
-                  if (need_mask && key > prm.L - prm.w + (ncol % prm.w)) pv = 0.0f;
+                for (int jj = 0; jj < 8; ++jj) {
+                  const int wi = wi0 + jj;
+                  float pv = fast_exp2(fmaf(__uint_as_float(sv[jj]), scale_log2, -lse_rows[ih * prm.w + (wi < 0 ? 0 : wi)]));
+                  if (wi < 0 || (need_mask && key > w0 + wi)) pv = 0.0f;
                   part += pv;
                 }
               }
@@ -687,7 +740,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             mbar_arrive(&mi.t_free[e]);
             if (b == 1) mi.xch[e][r] = part;
             named_barrier_sync(3, 256);
-            if (b == 0 && key < prm.L) {
+            if (b == 0 && key < len) {
               float* dst = prm.win_score + ((size_t)c * prm.Hkv + hkv) * prm.L + key;
               const float total = part + mi.xch[e][r];
               *dst = (u == 0) ? total : (*dst + total);
@@ -706,6 +759,10 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_before_sync();
   __syncthreads();
   if (warp == WARP_MMA) {
+    // no tensor-core operation may still be running when its accumulators are freed: both issuers ended with a
+    // commit to mma_done.  Immediate in a clean run; after an abort this is what makes the exit safe (the wait
+    // ignores the abort flag and is bounded).
+    mbar_wait_drain(&mi.mma_done, 0, cx.abort_flag);
     tc_fence_after_sync();
     tmem_dealloc(cx.tmem, 512);
   }
@@ -739,7 +796,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
   const int G = prm.Hq / prm.Hkv;
   const int n_items = prm.B * prm.Hkv * prm.n_rg * prm.n_split;
 
-  if (tid == 0) init_barriers(mi);
+  if (tid == 0) init_barriers(mi, prm.wait_kcycles);
   if (warp == WARP_MMA) tmem_alloc(&mi.tmem_base, 512);
   tc_fence_before_sync();
   __syncthreads();
@@ -811,6 +868,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
         const bool has_b = d.rows[b] > 0;
         mma_flash_block<D>(cx, wt, b, has_b, has_b ? d.n : 0, d.n, true);
       }
+      mma_commit(&mi.mma_done);
     }
     __syncwarp();
   } else if (warp < 8) {
@@ -888,6 +946,10 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
   tc_fence_before_sync();
   __syncthreads();
   if (warp == WARP_MMA) {
+    // no tensor-core operation may still be running when its accumulators are freed: both issuers ended with a
+    // commit to mma_done.  Immediate in a clean run; after an abort this is what makes the exit safe (the wait
+    // ignores the abort flag and is bounded).
+    mbar_wait_drain(&mi.mma_done, 0, cx.abort_flag);
     tc_fence_after_sync();
     tmem_dealloc(cx.tmem, 512);
   }

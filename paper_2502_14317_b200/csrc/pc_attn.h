@@ -10,11 +10,14 @@ namespace pc {
 struct PrefillParams {
   int C, L, w, Hq, Hkv;
   float scale_log2;              // softmax scale * log2(e)
+  const int* chunk_len;          // [C] tokens per chunk (window included) or null: all L
   float* lse;                    // [C,Hq,L] or null
   float* win_lse;                // [C,Hq,w]
   float* win_score;              // [C,Hkv,L]
   int* status;                   // device status word or null
   int* counter;                  // work-queue counter, zeroed before launch
+  int wait_kcycles;              // limit of every device-side wait, in units of 1024 cycles
+  int skip_final_publication;    // test hook of the bounded waits (see pc_debug_bounded_wait_test in pc.h)
 };
 
 // maps: rotated q (box 64x1x128x1), k_rot, v, o (store), rotated q with a w-row box
@@ -35,6 +38,7 @@ struct ParallelParams {
   float* lse_out;                // [B,Hq,w] or null
   int* status;
   int* counter;
+  int wait_kcycles;              // limit of every device-side wait, in units of 1024 cycles
 };
 
 // maps: q_win (w-row box), k_cache, v_cache (128-key box), k_win, v_win (128-row box over w tokens)

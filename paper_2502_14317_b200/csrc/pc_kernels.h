@@ -20,6 +20,10 @@ void launch_rope_table(double2* tab, float4* tab_hi, float4* tab_lo, int n_pos, 
 void launch_rope_rows(const void* x, const long long x_stride[3], void* y, const double2* tab, const float4* tab_hi,
                       const float4* tab_lo, int C, int L, int H, int d, cudaStream_t st);
 
+// Per-chunk lengths: zero o[c, p, :, :], lse[c, :, p] and win_score[c, :, p] for p >= clamp(chunk_len[c], w + 1, L).
+void launch_zero_chunk_tails(const int* chunk_len, int C, int L, int w, int Hq, int Hkv, int d, void* o,
+                             const long long o_stride[3], float* lse, float* win_score, cudaStream_t st);
+
 // ---- pc_select_gather.cu
 void launch_chunk_score(const float* win_lse, int C, int n_per_chunk, float* score, cudaStream_t st);
 void launch_select_chunks(const float* score, int C, int m, int lower_is_better, int* kept, cudaStream_t st);

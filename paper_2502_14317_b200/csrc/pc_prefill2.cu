@@ -58,8 +58,10 @@ struct __align__(16) Misc2 {
   uint64_t o_full, acc_free, lse_ready;
   uint64_t t_full[2], t_free[2];
   uint64_t m_pub[2][4];                      // [owner warpgroup][warp]: its reference maxima of a tile are in mref
+  uint64_t mma_done;                         // every tensor-core operation of the three issuers has completed (teardown)
   uint32_t tmem_base;
-  int abort_flag;
+  int abort_flag;                            // the two words after tmem_base stay adjacent: bounded waits read the limit
+  int wait_kcycles;                          // through the flag's address
   float lse2[1024];                          // window-row log-sum-exp (log2 units) of all G heads, G * w <= 1024
   float mref[2][TILE];                       // [tile parity][row]: reference maximum (log2 units) after that tile
   float xl[2][TILE];                         // [key half][row]: half-row sums
@@ -100,8 +102,12 @@ struct FastDiv {
   }
 };
 
+// With per-chunk lengths the query tiles of a shorter chunk are numbered from the END: slot v of the static
+// decomposition (v = T - 1 is the last tile of a full-length chunk) is tile v - (T - T_c) of a chunk with T_c tiles,
+// and slots below T - T_c are empty.  The window then always sits in the last one or two slots, which the tail item
+// of the group owns together with the score sweep.
 struct Sched2 {
-  int T, t_w, ntt, G, P, ipg, hp, n_pass;
+  int T, t_w, ntt, G, P, ipg, hp, n_pass, wp;
   FastDiv d_ipg, d_hkv, d_ntt, d_P;
 };
 __device__ __forceinline__ Sched2 make_sched2(const PrefillParams& p) {
@@ -109,10 +115,14 @@ __device__ __forceinline__ Sched2 make_sched2(const PrefillParams& p) {
   s.T = (p.L + TILE - 1) / TILE;
   s.G = p.Hq / p.Hkv;
   s.P = s.G / 2;
-  s.t_w = (p.L - p.w) / TILE;
-  s.ntt = s.T - s.t_w;
+  // slots of the tail item: the tiles that can hold window rows (with per-chunk lengths the window of some chunk
+  // may straddle two tiles even where that of a full-length chunk does not)
+  s.ntt = (p.chunk_len != nullptr) ? (p.w > 1 ? 2 : 1) : s.T - (p.L - p.w) / TILE;
+  if (s.ntt > s.T) s.ntt = s.T;
+  s.t_w = s.T - s.ntt;
   s.ipg = 1 + s.t_w * s.P;
-  const int cap = TILE / p.w, want = s.G / 2;
+  s.wp = (p.w + 7) & ~7;                                  // window rows of a head in the sweep operand (multiple of 8)
+  const int cap = TILE / s.wp, want = s.G / 2;
   s.hp = cap < want ? cap : want;                         // window heads per CTA and sweep pass
   s.n_pass = (s.G + 2 * s.hp - 1) / (2 * s.hp);
   s.d_ipg.init(s.ipg); s.d_hkv.init(p.Hkv); s.d_ntt.init(s.ntt); s.d_P.init(s.P);
@@ -127,15 +137,24 @@ struct Blk {
   int t;       // query tile of this CTA's block
   int n;       // key tiles the pair walks
 };
-__device__ __forceinline__ Blk decode_blk(const Sched2& s, int rank, int hkv, int within, int sub) {
+// length of chunk c in tokens (window included), clamped to (w, L]
+__device__ __forceinline__ int chunk_length(const PrefillParams& p, int c) {
+  if (p.chunk_len == nullptr) return p.L;
+  int len = __ldg(p.chunk_len + c);
+  len = len > p.L ? p.L : len;
+  return len <= p.w ? p.w + 1 : len;
+}
+// len: length of the block's chunk.  b.n == 0: an empty slot, every role skips the block.
+__device__ __forceinline__ Blk decode_blk(const Sched2& s, int rank, int hkv, int within, int sub, int len) {
   Blk b;
   const int h0 = hkv * s.G;
   int pair, tile;
   if (within == 0) { int rem; s.d_ntt.divmod(sub, pair, rem); tile = s.T - 1 - rem; }
   else { int q; s.d_P.divmod(within - 1, q, pair); tile = s.t_w - 1 - q; }
+  tile -= s.T - (len + TILE - 1) / TILE;
   b.h = h0 + 2 * pair + rank;
   b.t = tile;
-  b.n = tile + 1;
+  b.n = tile < 0 ? 0 : tile + 1;
   return b;
 }
 
@@ -161,7 +180,7 @@ __device__ __forceinline__ void mbar_wait_cluster(uint64_t* bar, uint32_t parity
   while (!mbar_try_wait_cluster(bar, parity)) {
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (clock64() - t0 > (static_cast<long long>(abort_flag[1]) << 10)) {
         *abort_flag = 1;
         if (status) atomicCAS(status, 0, where);
         return;
@@ -170,7 +189,7 @@ __device__ __forceinline__ void mbar_wait_cluster(uint64_t* bar, uint32_t parity
   }
 }
 
-__device__ __forceinline__ void init_barriers2(Misc2& mi) {
+__device__ __forceinline__ void init_barriers2(Misc2& mi, int wait_kcycles) {
   for (int b = 0; b < 2; ++b) {
     mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_free[b], 1);
     mbar_init(&mi.t_full[b], 1); mbar_init(&mi.t_free[b], 16);
@@ -184,7 +203,9 @@ __device__ __forceinline__ void init_barriers2(Misc2& mi) {
   mbar_init(&mi.pv_turn[0], 1); mbar_init(&mi.pv_turn[1], 1);
   mbar_init(&mi.o_full, 1); mbar_init(&mi.acc_free, 16); mbar_init(&mi.lse_ready, 16);
   for (int w = 0; w < 4; ++w) { mbar_init(&mi.m_pub[0][w], 1); mbar_init(&mi.m_pub[1][w], 1); }   // warp to warp (same rows)
+  mbar_init(&mi.mma_done, 3);
   mi.abort_flag = 0;
+  mi.wait_kcycles = wait_kcycles;
   fence_mbar_init();
 }
 
@@ -220,10 +241,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const Sched2 sch = make_sched2(prm);
   const int n_items = prm.C * prm.Hkv * sch.ipg;
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int n_sweep_tiles = (sch.T + 1) / 2;             // key tiles per CTA in the score sweep
-  const int rows_half = sch.hp * prm.w;                  // window rows per CTA and pass (B operand half)
+  const int rows_half = sch.hp * sch.wp;                 // sweep operand rows per CTA and pass (B operand half)
 
-  if (tid == 0) init_barriers2(mi);
+  if (tid == 0) init_barriers2(mi, prm.wait_kcycles);
   if (warp == WARP_QK) tmem_alloc_pair(&mi.tmem_base, 512);
   tc_fence_before_sync();
   __syncthreads();
@@ -242,8 +262,10 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         sch.d_ipg.divmod(item, group, within);
         sch.d_hkv.divmod(group, c, hkv);
         const int nsub = n_subitems2(sch, within);
+        const int len = chunk_length(prm, c);
         for (int sub = 0; sub < nsub; ++sub) {
-          const Blk bk = decode_blk(sch, rank, hkv, within, sub);
+          const Blk bk = decode_blk(sch, rank, hkv, within, sub, len);
+          if (bk.n == 0) continue;
           {
             const int qb = cQ & 1;
             WAIT2(&mi.q_free[qb], free_par(cQ >> 1), W2_QFREE);
@@ -272,7 +294,10 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
         if (within == 0) {
-          // ---- score sweep: window queries of hp heads per CTA and pass, then this CTA's key tiles
+          // ---- score sweep: window queries of hp heads per CTA and pass, then this CTA's key tiles.  A head's rows
+          // in the operand are the wp tokens that end with the chunk (wp = w rounded up to 8: the first wp - w rows
+          // are not window rows and are left out of the sums; a start before token 0 reads zeros)
+          const int n_sweep_tiles = ((len + TILE - 1) / TILE + 1) / 2;
           for (int u = 0; u < sch.n_pass; ++u) {
             const int qb = cQ & 1;
             WAIT2(&mi.q_free[qb], free_par(cQ >> 1), W2_QFREE);
@@ -282,8 +307,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               int g = u * 2 * sch.hp + (int)rank * sch.hp + i;
               if (g >= sch.G) g = sch.G - 1;              // filler rows: loaded, never summed
               for (int a = 0; a < 2; ++a)
-                tma_load_4d_pair(cx.sQ[qb] + a * 16384 + i * prm.w * 128, &tm_qw, bar, a * 64, hkv * sch.G + g,
-                                 prm.L - prm.w, c);
+                tma_load_4d_pair(cx.sQ[qb] + a * 16384 + i * sch.wp * 128, &tm_qw, bar, a * 64, hkv * sch.G + g,
+                                 len - sch.wp, c);
             }
             ++cQ;
             if (cK & 1) {                                 // a full key tile takes an even-aligned pair of stages
@@ -305,11 +330,19 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
       }
-      // every copy this CTA issued must have landed before it may exit: the last uses of the
-      // rings are consumed by the issuers, whose commits free the stages again
-      for (uint32_t i = (cK > NKS ? cK - NKS : 0); i < cK; ++i) WAIT2(&mi.k_free[i % NKS], full_par(i / NKS), W2_KFREE);
-      for (uint32_t i = (cV > NVS ? cV - NVS : 0); i < cV; ++i) WAIT2(&mi.v_free[i % NVS], full_par(i / NVS), W2_VFREE);
-      for (uint32_t i = (cQ > 2 ? cQ - 2 : 0); i < cQ; ++i) WAIT2(&mi.q_free[i & 1], full_par(i >> 1), W2_QFREE);
+      // Every copy issued must have landed before a CTA may exit.  In a run without a timed-out wait that follows
+      // from the last uses of the rings having been consumed (the teardown below waits for every tensor-core
+      // operation).  After an abort nothing is consumed any more: the leader, whose barriers count the bytes of both
+      // CTAs' copies, waits on them (ignoring the abort flag, bounded); the peer cannot observe the completion of
+      // its own last copies and lets a fixed pause pass that outlasts any copy in flight.
+      if (*cx.abort_flag) {
+        if (leader) {
+          for (uint32_t i = (cK > NKS ? cK - NKS : 0); i < cK; ++i) mbar_wait_drain(&mi.k_full[i % NKS], full_par(i / NKS), cx.abort_flag);
+          for (uint32_t i = (cV > NVS ? cV - NVS : 0); i < cV; ++i) mbar_wait_drain(&mi.v_full[i % NVS], full_par(i / NVS), cx.abort_flag);
+          for (uint32_t i = (cQ > 2 ? cQ - 2 : 0); i < cQ; ++i) mbar_wait_drain(&mi.q_full[i & 1], full_par(i >> 1), cx.abort_flag);
+        }
+        abort_grace_pause(cx.abort_flag);
+      }
     }
     __syncwarp();
   } else if (warp == WARP_QK) {
@@ -320,12 +353,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint32_t rk_u32 = smem_u32(cx.rK);
       uint32_t cQ = 0, cK = 0, cS = 0, cT = 0, n_done = 0;
       for (int item = pair_id; item < n_items; item += n_pairs) {
-        int group, within, c_unused, hkv;
+        int group, within, c, hkv;
         sch.d_ipg.divmod(item, group, within);
-        sch.d_hkv.divmod(group, c_unused, hkv);
+        sch.d_hkv.divmod(group, c, hkv);
         const int nsub = n_subitems2(sch, within);
+        const int len = chunk_length(prm, c);
         for (int sub = 0; sub < nsub; ++sub) {
-          const Blk bk = decode_blk(sch, rank, hkv, within, sub);
+          const Blk bk = decode_blk(sch, rank, hkv, within, sub, len);
+          if (bk.n == 0) continue;
           const int qb = cQ & 1;
           WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);           // the query tiles of both CTAs have landed
           ++cQ;
@@ -353,6 +388,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           // ---- score sweep.  Its two [128 keys x 256 rows] buffers overlay all of TMEM: every S/P
           // buffer is consumed and the accumulator has been read out once acc_free completes.
           WAIT2(&mi.acc_free, free_par(n_done), W2_ACCFREE);
+          const int n_sweep_tiles = ((len + TILE - 1) / TILE + 1) / 2;
           for (int u = 0; u < sch.n_pass; ++u) {
             const int qb = cQ & 1;
             WAIT2(&mi.q_full[qb], full_par(cQ >> 1), W2_QFULL);
@@ -388,6 +424,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           WAIT2(&mi.t_free[1], free_par(cT >> 1), W2_TFREE);
         }
       }
+      mma_commit_pair(&mi.mma_done);                         // teardown waits for everything this thread issued
     }
     __syncwarp();
   } else if (warp == WARP_PV || warp == WARP_PV + 1) {
@@ -401,12 +438,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint32_t rv_u32 = smem_u32(cx.rV);
       uint32_t cS = 0, n_done = 0, n_turn = 0;
       for (int item = pair_id; item < n_items; item += n_pairs) {
-        int group, within, c_unused, hkv;
+        int group, within, c, hkv;
         sch.d_ipg.divmod(item, group, within);
-        sch.d_hkv.divmod(group, c_unused, hkv);
+        sch.d_hkv.divmod(group, c, hkv);
         const int nsub = n_subitems2(sch, within);
+        const int len = chunk_length(prm, c);
         for (int sub = 0; sub < nsub; ++sub) {
-          const Blk bk = decode_blk(sch, rank, hkv, within, sub);
+          const Blk bk = decode_blk(sch, rank, hkv, within, sub, len);
+          if (bk.n == 0) continue;
           WAIT2(&mi.acc_free, free_par(n_done), W2_ACCFREE);                   // accumulator of the previous block read out
           for (int j = 0; j < bk.n; ++j, ++cS) {
             if ((int)(cS & 1) != me) continue;
@@ -436,6 +475,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           ++n_done;
         }
       }
+      mma_commit_pair(&mi.mma_done);
     }
     __syncwarp();
   } else if (warp < 8) {
@@ -464,8 +504,10 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       sch.d_ipg.divmod(item, group, within);
       sch.d_hkv.divmod(group, c, hkv);
       const int nsub = n_subitems2(sch, within);
+      const int len = chunk_length(prm, c);
       for (int sub = 0; sub < nsub; ++sub) {
-        const Blk bk = decode_blk(sch, rank, hkv, within, sub);
+        const Blk bk = decode_blk(sch, rank, hkv, within, sub, len);
+        if (bk.n == 0) continue;
         const int token = bk.t * TILE + r;
         const int qb = cQ & 1;                               // this block's query buffer (its output is staged there)
         ++cQ;
@@ -608,7 +650,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mi.xl[hlf][r] = l_run;
         named_barrier_sync(1, 256);
         const float l_tot = mi.xl[0][r] + mi.xl[1][r];
-        const float inv_l = 1.0f / l_tot;
+        const float inv_l = token < len ? 1.0f / l_tot : 0.0f;   // rows behind the end of the chunk are written as zeros
         {
           const uint32_t tO = cx.tmem + TM_O + hlf * 64 + lane_sel;
 #pragma unroll
@@ -621,7 +663,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               uint32_t pk[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e)
-                pk[e] = pack_bf16x2(__uint_as_float(o[g4 * 8 + 2 * e]) * inv_l, __uint_as_float(o[g4 * 8 + 2 * e + 1]) * inv_l);
+                pk[e] = token < len ? pack_bf16x2(__uint_as_float(o[g4 * 8 + 2 * e]) * inv_l, __uint_as_float(o[g4 * 8 + 2 * e + 1]) * inv_l) : 0u;
               *reinterpret_cast<uint4*>(myQ + hlf * 16384 + sw128_offset(r, q * 4 + g4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
           }
@@ -629,10 +671,10 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive_remote(a_acc_free);
-        if (hlf == 0 && token < prm.L) {
+        if (hlf == 0 && token < len) {
           const float lse2 = m_used + log2f(l_tot);
           if (prm.lse) prm.lse[((size_t)c * prm.Hq + bk.h) * prm.L + token] = lse2 * 0.6931471805599453f;
-          const int wi = token - (prm.L - prm.w);
+          const int wi = token - (len - prm.w);
           if (wi >= 0) {
             prm.win_lse[((size_t)c * prm.Hq + bk.h) * prm.w + wi] = lse2 * 0.6931471805599453f;
             if (within == 0) {                               // the sweep of both CTAs needs it
@@ -662,6 +704,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         mbar_wait_cluster(&mi.lse_ready, full_par(n_tail), cx.abort_flag, cx.status, W2_LSE);
         ++n_tail;
+        const int n_sweep_tiles = ((len + TILE - 1) / TILE + 1) / 2;
+        const int w0 = len - prm.w;                          // first window token of this chunk
         for (int u = 0; u < sch.n_pass; ++u) {
           const int qb = cQ & 1;                             // window queries of this pass (loaded and consumed by other warps)
           ++cQ;
@@ -672,20 +716,23 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             WAIT2(&mi.t_full[e], full_par(cT >> 1), W2_TFULL);
             tc_fence_after_sync();
             const int key = (2 * jj + (int)rank) * TILE + r;
-            const bool need_mask = (2 * jj + (int)rank) * TILE + TILE - 1 > prm.L - prm.w;
+            const bool need_mask = (2 * jj + (int)rank) * TILE + TILE - 1 > w0;
             const uint32_t tT = cx.tmem + e * 256 + hlf * rows_half + lane_sel;
             float part = 0.0f;
-            for (int c0 = 0; c0 < rows_half; c0 += 8) {
-              uint32_t sv[8];
-              tmem_ld8(tT + c0, sv);
-              tmem_wait_ld();
-              const int g = g_base + c0 / prm.w;             // w >= 8: the 8 columns belong to one head
-              if (g < sch.G) {
-                const float* lse_rows = mi.lse2 + g * prm.w + (c0 % prm.w);
+            for (int ih = 0; ih < sch.hp; ++ih) {            // heads of this column half; a head has wp columns, the last w are window rows
+              const int g = g_base + ih;
+              if (g >= sch.G) break;                         // filler head
+              const float* lse_head = mi.lse2 + g * prm.w;
+              for (int col = 0; col < sch.wp; col += 8) {
+                uint32_t sv[8];
+                tmem_ld8(tT + ih * sch.wp + col, sv);
+                tmem_wait_ld();
+                const int wi0 = col - (sch.wp - prm.w);      // window row of the first of these 8 columns (negative: not a window row)
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                  float pv = fast_exp2(fmaf(__uint_as_float(sv[i]), scale_log2, -lse_rows[i]));
-                  if (need_mask && key > prm.L - prm.w + (c0 % prm.w) + i) pv = 0.0f;
+                  const int wi = wi0 + i;
+                  float pv = fast_exp2(fmaf(__uint_as_float(sv[i]), scale_log2, -lse_head[wi < 0 ? 0 : wi]));
+                  if (wi < 0 || (need_mask && key > w0 + wi)) pv = 0.0f;
                   part += pv;
                 }
               }
@@ -695,7 +742,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (lane == 0) mbar_arrive_remote(map_to_cta(&mi.t_free[e], 0));
             mi.xs[e][hlf][r] = part;
             named_barrier_sync(1, 256);
-            if (hlf == 0 && key < prm.L) {
+            if (hlf == 0 && key < len) {
               float* dst = prm.win_score + ((size_t)c * prm.Hkv + hkv) * prm.L + key;
               const float total = part + mi.xs[e][1][r];
               *dst = (u == 0) ? total : (*dst + total);
@@ -716,6 +763,10 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   cluster_sync_all();
   if (warp == WARP_QK) {
+    // no tensor-core operation may still be running when its accumulators are freed: every issuer ended with a
+    // commit to mma_done (three arrivals in both CTAs).  Immediate in a clean run; after an abort this is what
+    // makes the exit safe.  The wait ignores the abort flag and is bounded.
+    mbar_wait_drain(&mi.mma_done, 0, cx.abort_flag);
     tc_fence_after_sync();
     tmem_dealloc_pair(cx.tmem, 512);
   }

@@ -84,4 +84,34 @@ void launch_rope_rows(const void* x, const long long x_stride[3], void* y, const
                                          tab_lo, tab, C, L, H, d);
 }
 
+// Rows behind the end of a chunk that is shorter than L (per-chunk lengths): outputs read as zero there.
+__global__ void zero_chunk_tails_kernel(const int* __restrict__ chunk_len, int L, int w, int Hq, int Hkv, int d,
+                                        uint16_t* __restrict__ o, long long so_chunk, long long so_tok, long long so_head,
+                                        float* __restrict__ lse, float* __restrict__ win_score) {
+  const int c = blockIdx.y;
+  int len = chunk_len[c];
+  len = len > L ? L : (len <= w ? w + 1 : len);
+  const int n_tail = L - len;
+  const long long per_tok = (long long)Hq * (d / 8);        // 16-byte pieces of an output row over all heads
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < (long long)n_tail * per_tok;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int p = len + (int)(i / per_tok), rest = (int)(i % per_tok), h = rest / (d / 8), piece = rest % (d / 8);
+    *reinterpret_cast<uint4*>(o + (long long)c * so_chunk + (long long)p * so_tok + (long long)h * so_head + piece * 8) =
+        make_uint4(0, 0, 0, 0);
+  }
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < (long long)n_tail * (Hq + Hkv);
+       i += (long long)gridDim.x * blockDim.x) {
+    const int row = (int)(i / n_tail), p = len + (int)(i % n_tail);
+    if (row < Hq) { if (lse != nullptr) lse[((size_t)c * Hq + row) * L + p] = 0.0f; }
+    else win_score[((size_t)c * Hkv + (row - Hq)) * L + p] = 0.0f;
+  }
+}
+
+void launch_zero_chunk_tails(const int* chunk_len, int C, int L, int w, int Hq, int Hkv, int d, void* o,
+                             const long long o_stride[3], float* lse, float* win_score, cudaStream_t st) {
+  note_launch();
+  zero_chunk_tails_kernel<<<dim3(64, (unsigned)C), 256, 0, st>>>(chunk_len, L, w, Hq, Hkv, d, (uint16_t*)o, o_stride[0],
+                                                                o_stride[1], o_stride[2], lse, win_score);
+}
+
 }  // namespace pc

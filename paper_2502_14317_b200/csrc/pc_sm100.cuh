@@ -2,11 +2,12 @@
 // mbarrier with bounded waits, TMA tiled copies, tcgen05 tensor-core MMA with
 // TMEM accumulators, and the shared-memory / instruction descriptors they take.
 //
-// Every wait here is bounded: after WAIT_LIMIT_CYCLES without completion the
-// waiter raises a CTA-wide abort flag; all later waits return at once, control
-// flow (which never depends on data) runs to its normal end, and the host sees
-// PC_ERR_TIMEOUT in the status word.  A bug in a barrier phase therefore cannot
-// leave the GPU spinning.
+// Every wait here is bounded: after the wait limit (about a second by default) without
+// completion the waiter raises a CTA-wide abort flag and stores a code that names the
+// wait in the caller's status word; all later waits return at once, control flow (which
+// never depends on data) runs to its normal end, copies and tensor-core work in flight
+// are drained, and the kernel returns.  A bug in a barrier phase therefore cannot leave
+// the GPU spinning.
 #pragma once
 #include <cstdint>
 #include <cuda_bf16.h>
@@ -14,11 +15,8 @@
 
 namespace pc {
 
-constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // ~1 s at B200 clocks
-#ifndef PC_SPIN_BACKOFF_NS
-#define PC_SPIN_BACKOFF_NS 20
-#endif
-constexpr unsigned SPIN_BACKOFF_NS = PC_SPIN_BACKOFF_NS;   // pause between two polls of a barrier (0: none)
+constexpr int WAIT_LIMIT_KCYCLES = 1 << 21;              // default wait limit in units of 1024 cycles: ~1 s at B200 clocks
+constexpr unsigned SPIN_BACKOFF_NS = 20;                 // pause between two polls of a barrier
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -50,9 +48,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  `abort_flag` lives in shared memory; once it is non-zero every
-// wait returns immediately (the result data is then garbage and the status word
-// says so).  Returns false if the wait gave up.
+// Bounded wait.  `abort_flag` points at two adjacent ints in shared memory: the CTA's abort
+// flag and the wait limit in units of 1024 cycles.  Once the flag is non-zero every wait
+// returns immediately (the result data is then garbage and the status word says so).
+// Returns false if the wait gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           int* status_word, int where) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -63,7 +62,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (SPIN_BACKOFF_NS > 0) __nanosleep(SPIN_BACKOFF_NS);   // a hot spin takes issue slots from the warps that share the scheduler
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (clock64() - t0 > (static_cast<long long>(abort_flag[1]) << 10)) {
         *abort_flag = 1;
         if (status_word) atomicCAS(status_word, 0, where);
         return false;
@@ -72,12 +71,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   }
 }
 
-// Wait that ignores the abort flag (used only to drain copies in flight before exit).
-__device__ __forceinline__ void mbar_wait_drain(uint64_t* bar, uint32_t parity) {
+// Wait that ignores the abort flag (used only to drain copies and tensor-core work in flight before
+// exit); gives up after an eighth of the wait limit.
+__device__ __forceinline__ void mbar_wait_drain(uint64_t* bar, uint32_t parity, const volatile int* abort_flag) {
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES / 8) return;
+    if (clock64() - t0 > (static_cast<long long>(abort_flag[1]) << 7)) return;
   }
+}
+// After an abort: a fixed pause (a tenth of a millisecond) that outlasts any copy this CTA may still have in
+// flight towards its shared memory whose completion it cannot observe on a barrier of its own.
+__device__ __forceinline__ void abort_grace_pause(const volatile int* abort_flag) {
+  if (*abort_flag == 0) return;
+  const long long t0 = clock64();
+  while (clock64() - t0 < 200000LL) __nanosleep(1000);
 }
 
 // ------------------------------------------------------------------ fences

@@ -53,7 +53,9 @@ def test_workspace_queries_are_host_only(lib):
     with_krot = binding.chunk_prefill_attn_workspace_bytes(16, 8192, 64, 32, 8, 128, k_rot_in_workspace=True)
     assert with_krot == tables(8192, 128) + 16 * 8192 * 32 * 128 * 2 + 16 * 8192 * 8 * 128 * 2
     # unsupported shapes give 0
-    assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 24, 4, 2, 64) == 0       # window not a power of two
+    assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 24, 4, 2, 64) > 0        # any window up to 128 tokens
+    assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 129, 4, 2, 64) == 0      # wider than a tile
+    assert binding.chunk_prefill_attn_workspace_bytes(1, 64, 64, 4, 2, 64) == 0        # no context token left
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 2, 96) == 0       # head size
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 3, 64) == 0       # Hq % Hkv
     assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 128, 16384) > 0
@@ -69,13 +71,15 @@ def test_host_side_argument_errors_need_no_gpu(lib):
     assert lib.pc_select_chunks(p, 4, 5, 1, o, None) == -1          # m > C
     assert lib.pc_select_chunks(p, 2000, 5, 1, o, None) == -2       # C > 1024
     assert lib.pc_select_tokens(p, o, 4, 2, 2, 256, 300, 64, o, None) == -1    # n_cand > L
-    assert lib.pc_gather_kv(p, p, None, 256, o, o, 2, 2, 64, 96, p, p, None, None) == -2   # head size
+    st = (ctypes.c_int64 * 3)(256 * 2 * 96, 2 * 96, 96)
+    assert lib.pc_gather_kv(p, p, st, o, o, 2, 2, 64, 96, p, p, None, None) == -2   # head size
+    assert lib.pc_gather_kv(p, p, None, o, o, 2, 2, 64, 64, p, p, None, None) == -1  # no strides
     assert lib.pc_parallel_attn(1, 24, 4, 2, 64, 128, p, 0, 1e4, 0.0, p, p, p, p, p, None, None, None, 0, None) == -2
     assert lib.pc_select_tokens_calibrated(p, o, 4, 2, 2, 256, 200, 64, -1, 0, 1.0, 1.0, 1.0, o, None) == -1   # n_s < 0
     assert lib.pc_queue_init(0, p, o, None) == -1                    # no slots
     assert lib.pc_queue_update(p, 4, -1, 1, 2, p, o, o, None) == -1  # negative chunk id
     assert lib.pc_queue_update(p, 1000, 0, 1, 100, p, o, o, None) == -2   # slots + batch > 1024
-    assert lib.pc_queue_gather(p, p, None, 256, o, o, 2, 2, 64, 96, p, p, o, None) == -2   # head size
+    assert lib.pc_queue_gather(p, p, st, o, o, 2, 2, 64, 96, p, p, o, None) == -2   # head size
     assert lib.pc_queue_emit(o, 2, 2, 64, 128, p, p, o, o, None, p, p, None, None) == -1    # no slot_order array
 
 
@@ -143,3 +147,34 @@ def test_bench_without_launcher_starts_its_own_ranks():
     code = "import os, sys; sys.exit(0 if os.environ['WORLD_SIZE'] == '2' and os.environ['RANK'] in '01' else 7)"
     assert bench.spawn_workers([sys.executable, "-c", code], 2) == 0
     assert bench.spawn_workers([sys.executable, "-c", "import os, sys; sys.exit(5 * int(os.environ['RANK']))"], 2) == 5
+
+
+def _params(name):
+    """Parameter names of the prototype of `name` in include/pc.h, in order."""
+    text = open(os.path.join(ROOT, "include", "pc.h")).read()
+    m = re.search(r"PC_API\s+[\w\s\*]+?\b" + name + r"\s*\(([^;]*?)\)\s*;", text, re.S)
+    assert m, name
+    out = []
+    for piece in m.group(1).replace("\n", " ").split(","):
+        piece = piece.strip()
+        if piece in ("void", ""):
+            continue
+        out.append(re.sub(r"\[\d*\]$", "", piece).split()[-1].lstrip("*"))
+    return out
+
+
+def test_boundary_has_the_argument_lists_of_the_scope_table():
+    """The five calls of the path: argument names and order as the scope table lists them.  Two documented
+    additions: the optional full log-sum-exp output `lse` of the prefill call, and `Hkv` in the parallel-attention
+    workspace query (the split plan depends on the number of kv-heads)."""
+    assert _params("pc_chunk_prefill_attn_workspace_bytes") == ["desc"]
+    assert _params("pc_chunk_prefill_attn") == ["desc", "q", "k", "v", "chunk_len", "o", "k_rot", "lse", "win_score",
+                                                "win_lse", "status_word", "workspace", "workspace_bytes", "stream"]
+    assert _params("pc_select_chunks") == ["chunk_score", "C", "m", "lower_is_better", "kept", "stream"]
+    assert _params("pc_select_tokens") == ["win_score", "kept", "C", "m", "Hkv", "L", "n_cand", "k", "idx", "stream"]
+    assert _params("pc_gather_kv") == ["k_src", "v_src", "kv_stride", "kept", "idx", "m", "Hkv", "k", "d", "k_out",
+                                       "v_out", "pos_out", "stream"]
+    assert _params("pc_parallel_attn_workspace_bytes") == ["B", "w", "Hq", "Hkv", "d", "Nk"]
+    assert _params("pc_parallel_attn") == ["B", "w", "Hq", "Hkv", "d", "Nk", "q_win", "q_pos0", "rope_theta",
+                                           "softmax_scale", "k_cache", "v_cache", "k_win", "v_win", "out", "lse_out",
+                                           "status_word", "workspace", "workspace_bytes", "stream"]

@@ -54,6 +54,16 @@ def test_cfg0_full(cfg0_inputs):
     (2, 1100, 64, 6, 2, 128, 10000.0),     # G=3 (odd): tile-pair mode, 9 tiles, ragged
     (1, 1024, 8, 2, 2, 128, 10000.0),      # MHA, even tile count, smallest window
     (1, 200, 128, 8, 1, 128, 10000.0),     # G*w = 1024 window rows: four score passes, window over two tiles
+    # windows that are no power of two (the sweep pads a head's rows to a multiple of 8 and leaves the pad out)
+    (2, 400, 24, 4, 2, 128, 10000.0),      # CTA pairs, w = 24
+    (1, 700, 100, 4, 1, 128, 500000.0),    # CTA pairs, w = 100 (the region size of App. C), window over two tiles
+    (1, 300, 5, 2, 1, 128, 10000.0),       # CTA pairs, w = 5 < 8
+    (1, 260, 1, 4, 2, 128, 10000.0),       # CTA pairs, a single query token
+    (2, 400, 24, 3, 3, 128, 10000.0),      # multi-head (single-CTA kernel, tile-pair mode), w = 24
+    (1, 520, 100, 6, 2, 128, 10000.0),     # G = 3, w = 100
+    (2, 300, 24, 4, 2, 64, 10000.0),       # head size 64, w = 24
+    (1, 333, 100, 2, 1, 64, 10000.0),      # head size 64, w = 100
+    (1, 140, 3, 8, 2, 64, 10000.0),        # head size 64, w = 3
 ])
 def test_shapes(C, L, w, Hq, Hkv, d, theta):
     rng = np.random.default_rng(L * 7 + Hq)
@@ -129,7 +139,7 @@ def test_argument_errors():
     q = torch.zeros((1, 256, 4, 64), dtype=torch.bfloat16, device="cuda")
     k = torch.zeros((1, 256, 2, 64), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(pc.PcError, match="unsupported"):
-        pc.chunk_prefill_attn(q, k, k, w=24, rope_theta=1e4)           # window not a power of two
+        pc.chunk_prefill_attn(q, k, k, w=129, rope_theta=1e4)          # window wider than a tile
     with pytest.raises(pc.PcError, match="invalid"):
         pc.chunk_prefill_attn(q, k, k, w=256, rope_theta=1e4)          # window >= L
     q96 = torch.zeros((1, 256, 4, 96), dtype=torch.bfloat16, device="cuda")
@@ -145,10 +155,10 @@ def test_argument_errors():
     ws = torch.empty(64, dtype=torch.uint8, device="cuda")
     S = torch.empty((1, 2, 256), dtype=torch.float32, device="cuda")
     Lw = torch.empty((1, 4, 16), dtype=torch.float32, device="cuda")
-    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(k), _ptr(o), None, None, _ptr(S), _ptr(Lw),
+    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(k), None, _ptr(o), None, None, _ptr(S), _ptr(Lw),
                                    None, _ptr(ws), ws.numel(), None)
     assert rc == -3                                                     # PC_ERR_WORKSPACE
-    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), None, _ptr(k), _ptr(k), _ptr(o), None, None, _ptr(S), _ptr(Lw),
+    rc = lib.pc_chunk_prefill_attn(ctypes.byref(desc), None, _ptr(k), _ptr(k), None, _ptr(o), None, None, _ptr(S), _ptr(Lw),
                                    None, _ptr(ws), ws.numel(), None)
     assert rc == -1                                                     # PC_ERR_INVALID_ARG
 
@@ -174,3 +184,80 @@ def test_rope_position_reuse_equals_fp64_rotation_rounded_once(C, L, H, d, theta
     ref = orc.rope_bf16(bits, theta)
     bad = np.argwhere(got != ref)
     assert bad.shape[0] == 0, f"{bad.shape[0]} of {ref.size} rotated values differ from the fp64 rotation, first at {bad[0]}"
+
+
+@pytest.mark.parametrize("L,w,Hq,Hkv,d,lens", [
+    (640, 64, 4, 2, 128, [640, 500, 129, 65, 384]),      # CTA pairs: full, ragged, two tiles, one tile, tile-aligned
+    (520, 24, 4, 1, 128, [300, 520, 25, 256]),           # w = 24, the shortest chunk has a single context token
+    (640, 64, 3, 3, 128, [640, 333, 130, 65]),           # multi-head, single-CTA kernel (tile-pair mode)
+    (400, 16, 4, 2, 64, [400, 17, 250, 128]),            # head size 64
+    (300, 100, 2, 2, 64, [101, 300, 229]),               # head size 64, multi-head, w = 100
+])
+def test_chunks_of_different_lengths_in_one_call(L, w, Hq, Hkv, d, lens):
+    """Sec. 3.1: chunks of AT MOST the trained length.  chunk_len[c] tokens of chunk c count (window included, the
+    window directly behind the context); every chunk must equal the oracle run on that chunk alone, and everything
+    at or behind its end reads as zero."""
+    import paper_2502_14317_b200 as pc
+    C = len(lens)
+    rng = np.random.default_rng(L + w + Hq + d)
+    q = pc_inputs.f32_to_bf16_bits(rng.standard_normal((C, L, Hq, d)).astype(np.float32))
+    k = pc_inputs.f32_to_bf16_bits(rng.standard_normal((C, L, Hkv, d)).astype(np.float32))
+    v = pc_inputs.f32_to_bf16_bits(rng.standard_normal((C, L, Hkv, d)).astype(np.float32))
+    k[:, 0] = pc_inputs.f32_to_bf16_bits(pc_inputs.bf16_bits_to_f32(k[:, 0]) * np.float32(4.0))
+    theta, G = 10000.0, Hq // Hkv
+    cl = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    nan = float("nan")
+    res = pc.chunk_prefill_attn(to_dev(q), to_dev(k), to_dev(v), w=w, rope_theta=theta, want_lse=True, chunk_len=cl,
+                                out=torch.full((C, L, Hq, d), nan, dtype=torch.bfloat16, device="cuda"),
+                                win_score=torch.full((C, Hkv, L), nan, dtype=torch.float32, device="cuda"),
+                                lse=torch.full((C, Hq, L), nan, dtype=torch.float32, device="cuda"))
+    torch.cuda.synchronize()
+    assert int(res["status"].item()) == 0
+    got_o, got_S = to_f64(res["o"]), res["win_score"].cpu().numpy()
+    got_lse, got_wl = res["lse"].cpu().numpy().astype(np.float64), res["win_lse"].cpu().numpy().astype(np.float64)
+    assert np.array_equal(to_bits(res["k_rot"]), orc.rope_bf16(k, theta))
+    scale = 1.0 / np.sqrt(d)
+    for c, n in enumerate(lens):
+        qc, kc, vc = q[c:c + 1, :n], k[c:c + 1, :n], v[c:c + 1, :n]
+        O, LSE, k_rot = orc.local_attention(qc, kc, vc, theta)
+        S, _, LSE_win = orc.window_scores(orc.rope_bf16(qc, theta), k_rot, vc, w, scale)
+        check_attention_output(got_o[c:c + 1, :n], O, f"O of chunk {c} ({n} tokens)")
+        assert np.abs(got_lse[c:c + 1, :, :n] - LSE).max() <= 2e-3
+        assert np.abs(got_wl[c:c + 1] - LSE_win).max() <= 2e-3
+        check_scores(got_S[c:c + 1, :, :n], S, G, w, n)
+        assert np.allclose(got_S[c, :, :n].sum(-1), G * w, rtol=1e-4)
+        assert np.all(got_o[c, n:] == 0.0) and np.all(got_S[c, :, n:] == 0.0) and np.all(got_lse[c, :, n:] == 0.0)
+
+
+def test_a_wait_that_runs_out_returns_a_status_and_leaves_the_device_usable(cfg0_inputs):
+    """Every device-side wait is bounded.  Here one is made to run out without faulting anything: the producer
+    warp of the single-CTA kernel (head size 64) leaves out the data-free "no more work" signal after the last
+    work item, when no copy and no tensor-core operation is in flight; the consumer warps wait for it for about a
+    millisecond (limit set through the test hook), store the code of that wait in the status word, drain and
+    return.  The outputs of that call are complete, and the next call on the same stream is bit-identical to a
+    clean run."""
+    import paper_2502_14317_b200 as pc
+    cfg, inp = cfg0_inputs
+    q, k, v = to_dev(inp["q"]), to_dev(inp["k"]), to_dev(inp["v"])
+    lib = pc.load_library()
+
+    def run():
+        r = pc.chunk_prefill_attn(q, k, v, w=cfg.w, rope_theta=cfg.rope_theta, want_lse=True)
+        torch.cuda.synchronize()
+        return r
+
+    clean = run()
+    assert int(clean["status"].item()) == 0
+    assert lib.pc_debug_bounded_wait_test(2_000_000, 1) == 0          # waits give up after 2e6 cycles (about 1 ms)
+    try:
+        hit = run()
+    finally:
+        assert lib.pc_debug_bounded_wait_test(0, 0) == 0
+    code = int(hit["status"].item())
+    assert code == 101, f"expected the code of the work-item wait in the status word, got {code}"
+    for key in ("o", "win_score", "win_lse", "lse", "k_rot"):
+        assert torch.equal(hit[key], clean[key]), key                 # all work was done before the missing signal
+    again = run()
+    assert int(again["status"].item()) == 0
+    for key in ("o", "win_score", "win_lse", "lse", "k_rot"):
+        assert torch.equal(again[key], clean[key]), key
