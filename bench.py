@@ -139,7 +139,9 @@ def run_reference(args, cfg):
             "config": workload_description(cfg),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-            "gpu_launches": 0}
+            "gpu_launches": 0,
+            "note": "steps and warmup are capped at 3 and 1 for this arm (one oracle sample takes about ten seconds); "
+                    "the GPU arm runs the step counts it was given"}
     print(json.dumps(line))
 
 
@@ -274,8 +276,8 @@ def run_gpu(args, cfg):
                                     win_lse=buffers.get("win_lse"), status=buffers.get("status"),
                                     workspace=buffers.get("ws_prefill"))
         if events: events[1].record()
-        score = pc.chunk_score_from_lse(pre["win_lse"], out=buffers.get("chunk_score"))
-        kept = pc.select_chunks(score, cfg.m, True, out=buffers.get("kept"))
+        score, kept = pc.score_select_chunks(pre["win_lse"], cfg.m, True, score_out=buffers.get("chunk_score"),
+                                             kept_out=buffers.get("kept"))
         idx = pc.select_tokens(pre["win_score"], kept, L - w, cfg.k, out=buffers.get("idx"))
         if events: events[2].record()
         kc, vc, pos = pc.gather_kv(pre["k_rot"], v, kept, idx, k_out=buffers.get("kc"), v_out=buffers.get("vc"),
@@ -289,10 +291,9 @@ def run_gpu(args, cfg):
                        kc=kc, vc=vc, pos=pos, fg=pa["out"], ws_par=pa["workspace"])
         return pa["out"]
 
-    # kernels launched by one step: rope table, rope keys, prefill attention, chunk score, chunk top-m,
-    # token top-k, gather, rope table (window), parallel attention, split merge
-    n_split_merge = 1 if pc.parallel_attn_workspace_bytes(1, w, cfg.Hq, cfg.Hkv, cfg.d, cfg.m * cfg.k) > 65536 else 0
-    launches_per_step = 9 + n_split_merge
+    # kernels of one step (counted by the library, see pc_launch_count): cos/sin table, rotation of keys and of
+    # queries, chunk attention, stand-in score + chunk top-m, token top-k, gather, window cos/sin table, parallel
+    # attention, merge of its key splits
 
     def barrier():
         torch.cuda.synchronize()
@@ -314,6 +315,7 @@ def run_gpu(args, cfg):
     barrier()
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
+    launches_before = pc.launch_count()
     t_start.record()
     for s in range(args.steps):
         ev[s][0].record()
@@ -322,11 +324,21 @@ def run_gpu(args, cfg):
     t_end.record()
     barrier()
     total_ms = t_start.elapsed_time(t_end)
+    launches_timed = pc.launch_count() - launches_before
     clocks = sampler.stop() if sampler else None
     assert int(buffers["status"].item()) == 0, "a device-side wait ran out"
 
     stage_ms = {name: statistics.mean(ev[s][a].elapsed_time(ev[s][b]) for s in range(args.steps))
                 for name, a, b in (("prefill_attn", 0, 1), ("score_select", 1, 2), ("gather", 2, 3), ("parallel_attn", 3, 4))}
+
+    # ---- launch floor of the ranking stage: two launches that do (next to) nothing, timed like the stage
+    tiny_lse = torch.zeros((1, 1, 1), dtype=torch.float32, device=dev)
+    tiny_buf = {}
+
+    def two_tiny_launches():
+        tiny_buf["s"], tiny_buf["k"] = pc.score_select_chunks(tiny_lse, 1, True, score_out=tiny_buf.get("s"), kept_out=tiny_buf.get("k"))
+        tiny_buf["s"], tiny_buf["k"] = pc.score_select_chunks(tiny_lse, 1, True, score_out=tiny_buf.get("s"), kept_out=tiny_buf.get("k"))
+    empty_pair_ms = _time_us(torch, two_tiny_launches, warm=3, reps=50) / 1e3
 
     # ---- end to end through the public API with host buffers: H2D of Q,K,V and D2H of the result every step
     e2e_steps = max(1, min(args.steps, 5))
@@ -385,7 +397,7 @@ def run_gpu(args, cfg):
             "e2e": {"value": replica_throughput(tokens, world, e2e_ms), "unit": UNIT,
                     "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
                     "d2h_bytes_per_step": int(h_out.numel()) * 2, "ms_per_step": e2e_ms, "steps": e2e_steps},
-            "gpu_launches": launches_per_step * args.steps,
+            "gpu_launches": launches_timed,
             "roofline": {"bound": "tensor", "kernel": ("prefill_pair_kernel" if pair_path else "prefill_attn_kernel") +
                                    " (+ RoPE table and key pre-pass inside the same call)",
                          "achieved": ach_tflops, "peak": peak_tflops, "unit": "TFLOP/s",
@@ -401,7 +413,9 @@ def run_gpu(args, cfg):
                 "prefill_attn": {"ms": stage_ms["prefill_attn"], "tflops": ach_tflops},
                 "score_select": {"ms": stage_ms["score_select"], "algorithmic_bytes": sel_bytes,
                                  "gbs": sel_bytes / (stage_ms["score_select"] * 1e-3) / 1e9,
-                                 "note": "three launches (chunk score, chunk top-m, token top-k); latency-bound at this size"},
+                                 "launches": 2, "launch_floor_ms": empty_pair_ms,
+                                 "note": "two launches (stand-in score + chunk top-m; token top-k), latency-bound at this size; "
+                                         "launch_floor_ms = two empty kernels timed the same way"},
                 "gather": {"ms": stage_ms["gather"], "algorithmic_bytes": gather_bytes,
                            "gbs": gather_bytes / (stage_ms["gather"] * 1e-3) / 1e9,
                            "frac_of_measured_hbm": gather_bytes / (stage_ms["gather"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
@@ -458,15 +472,41 @@ def streamed_measurement(pc, torch, cfg, q, k, v, step_buffers, batch=4) -> dict
                     "pc_queue_emit + pc_parallel_attn at the end; same results as the timed step"}
 
 
-def extra_measurements(pc, torch, dev, peaks, only=None, select_chunks=8192) -> dict:
+def _extra_prefill(pc, torch, dev, peaks, g, out):
+    """pc_chunk_prefill_attn at the two other full-size shapes (one call each, random device data)."""
+    for name in ("cfg2", "cfg3"):
+        cfg = pc_inputs.get_config(name)
+        q = torch.randn((cfg.C, cfg.L, cfg.Hq, cfg.d), device=dev, generator=g).bfloat16()
+        k = torch.randn((cfg.C, cfg.L, cfg.Hkv, cfg.d), device=dev, generator=g).bfloat16()
+        v = torch.randn((cfg.C, cfg.L, cfg.Hkv, cfg.d), device=dev, generator=g).bfloat16()
+        buf = {}
+
+        def run():
+            r = pc.chunk_prefill_attn(q, k, v, w=cfg.w, rope_theta=cfg.rope_theta, out=buf.get("o"), k_rot=buf.get("k_rot"),
+                                      win_score=buf.get("win_score"), win_lse=buf.get("win_lse"), status=buf.get("status"),
+                                      workspace=buf.get("workspace"))
+            buf.update(r)
+        us = _time_us(torch, run, warm=3, reps=5)
+        assert int(buf["status"].item()) == 0
+        tf = prefill_flops(cfg) / us / 1e6
+        out["prefill_" + name] = {"us": us, "tflops": tf, "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"],
+                                  "kernel": "prefill_pair_kernel" if (cfg.d == 128 and cfg.G % 2 == 0) else "prefill_attn_kernel",
+                                  "workload": workload_description(cfg)["workload"]}
+        del q, k, v, buf
+        torch.cuda.empty_cache()
+
+
+def extra_measurements(pc, torch, dev, peaks, only=None, select_chunks=8192, parallel_batch=64) -> dict:
     """Single-call timings of the stages whose full-size workloads are not part of the cfg1 step
     (outside the timed region; random device data, parity is covered by the tests):
     parallel attention over a batch of compressed caches (cfg4), token top-k on enough rows to be
     bandwidth-bound, and the gather at the cfg2 size."""
     out = {}
     g = torch.Generator(device=dev).manual_seed(4)
+    if only in (None, "prefill"):
+        _extra_prefill(pc, torch, dev, peaks, g, out)
     if only in (None, "parallel"):
-        _extra_parallel(pc, torch, dev, peaks, g, out)
+        _extra_parallel(pc, torch, dev, peaks, g, out, parallel_batch)
     if only in (None, "select"):
         _extra_select(pc, torch, dev, peaks, g, out, select_chunks)
     if only in (None, "gather"):
@@ -474,9 +514,9 @@ def extra_measurements(pc, torch, dev, peaks, only=None, select_chunks=8192) -> 
     return out
 
 
-def _extra_parallel(pc, torch, dev, peaks, g, out):
-    # ---- cfg4: B=64 sequences x (8 kept chunks x 2048 keys), 64 window queries
-    B, w, Hq, Hkv, d, Nk = 64, 64, 32, 8, 128, 16384
+def _extra_parallel(pc, torch, dev, peaks, g, out, B=64):
+    # ---- cfg4: B=64 sequences x (8 kept chunks x 2048 keys), 64 window queries (a smaller B for an ncu capture)
+    w, Hq, Hkv, d, Nk = 64, 32, 8, 128, 16384
     qw = torch.randn((B, w, Hq, d), device=dev, generator=g).bfloat16()
     kc = torch.randn((B, Hkv, Nk, d), device=dev, generator=g).bfloat16()
     vc = torch.randn((B, Hkv, Nk, d), device=dev, generator=g).bfloat16()
@@ -491,7 +531,7 @@ def _extra_parallel(pc, torch, dev, peaks, g, out):
     us = _time_us(torch, run_par, reps=10)
     flops = 4.0 * d * (Nk + (w + 1) / 2) * w * Hq * B
     kv_bytes = 2.0 * B * Hkv * Nk * d * 2
-    out["parallel_attn_cfg4"] = {"us": us, "tflops": flops / us / 1e6, "kv_gbs": kv_bytes / us / 1e3,
+    out["parallel_attn_cfg4" if B == 64 else "parallel_attn_cfg4_B%d" % B] = {"us": us, "tflops": flops / us / 1e6, "kv_gbs": kv_bytes / us / 1e3,
                                  "frac_of_measured_bf16_burst": flops / us / 1e6 / peaks["bf16_tflops"],
                                  "frac_of_measured_hbm": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
                                  "flops": flops, "kv_bytes": kv_bytes, "l2": "4.3 GB of K/V per call, larger than L2"}
@@ -551,7 +591,9 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the single-call timings of cfg4 / scaled select / cfg2 gather")
-    ap.add_argument("--extra-only", default=None, choices=["parallel", "select", "gather"],
+    ap.add_argument("--parallel-batch", type=int, default=64,
+                    help="sequences of the parallel-attention measurement (smaller for an ncu capture)")
+    ap.add_argument("--extra-only", default=None, choices=["parallel", "select", "gather", "prefill"],
                     help="run only that single-call measurement and print it (no step loop; e.g. for an ncu capture)")
     ap.add_argument("--select-chunks", type=int, default=8192,
                     help="rows / 8 of the scaled token top-k measurement (smaller for an ncu capture)")
@@ -571,7 +613,7 @@ def main():
         dev = torch.device("cuda:0")
         torch.cuda.set_device(dev)
         print(json.dumps({"extra": extra_measurements(pc, torch, dev, load_peaks(), only=args.extra_only,
-                                                      select_chunks=args.select_chunks)}))
+                                                      select_chunks=args.select_chunks, parallel_batch=args.parallel_batch)}))
         return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # started without a launcher: become the launcher of --gpus replicas, one process per GPU

@@ -164,6 +164,15 @@ PC_API int32_t pc_select_chunks(const float* chunk_score, int32_t C, int32_t m, 
                          int32_t* kept, void* stream);
 
 /* ------------------------------------------------------------------------------------
+ * pc_chunk_score_from_lse followed by pc_select_chunks (same results, bit for bit) as one
+ * call: for up to 64 chunks a single launch, which matters where the whole ranking stage
+ * moves a few megabytes and is bound by launch latency.  Used by the synthetic single-layer
+ * pipeline only (the stand-in score is not part of the paper).
+ */
+PC_API int32_t pc_score_select_chunks(const float* win_lse, int32_t C, int32_t Hq, int32_t w, int32_t m,
+                                int32_t lower_is_better, float* chunk_score, int32_t* kept, void* stream);
+
+/* ------------------------------------------------------------------------------------
  * Token eviction per kept chunk and kv-head.  Paper: Sec. 3.1 "Parallel KV cache
  * eviction", Eq. 7.
  * For row (r, hkv), r < m: the k largest of win_score[kept[r], hkv, 0..n_cand) (window

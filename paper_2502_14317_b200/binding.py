@@ -58,6 +58,8 @@ def load_library():
     lib.pc_launch_count.argtypes = []
     lib.pc_chunk_score_from_lse.restype = c_int32
     lib.pc_chunk_score_from_lse.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
+    lib.pc_score_select_chunks.restype = c_int32
+    lib.pc_score_select_chunks.argtypes = [c_void_p] + [c_int32] * 5 + [c_void_p, c_void_p, c_void_p]
     lib.pc_select_chunks.restype = c_int32
     lib.pc_select_chunks.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
     lib.pc_select_tokens.restype = c_int32
@@ -212,6 +214,18 @@ def select_chunks(chunk_score, m, lower_is_better=True, out=None):
     _check(lib.pc_select_chunks(_ptr(chunk_score), C, int(m), int(bool(lower_is_better)), _ptr(out), _stream()),
            "pc_select_chunks")
     return out
+
+
+def score_select_chunks(win_lse, m, lower_is_better=True, score_out=None, kept_out=None):
+    """pc_score_select_chunks: win_lse [C,Hq,w] fp32 -> (chunk_score [C] fp32, kept [m] int32), one launch for C <= 64."""
+    lib = load_library()
+    _need_cuda(win_lse)
+    C, Hq, w = win_lse.shape
+    score = torch.empty(C, dtype=torch.float32, device=win_lse.device) if score_out is None else score_out
+    kept = torch.empty(m, dtype=torch.int32, device=win_lse.device) if kept_out is None else kept_out
+    _check(lib.pc_score_select_chunks(_ptr(win_lse), C, Hq, w, int(m), int(bool(lower_is_better)), _ptr(score), _ptr(kept),
+                                      _stream()), "pc_score_select_chunks")
+    return score, kept
 
 
 def select_tokens(win_score, kept, n_cand, k, out=None):
@@ -394,8 +408,10 @@ def hot_path(q, k, v, *, w, rope_theta, m, k_keep, softmax_scale=0.0, chunk_scor
     pre = chunk_prefill_attn(q, k, v, w=w, rope_theta=rope_theta, softmax_scale=softmax_scale, out=b.get("o"),
                              k_rot=b.get("k_rot"), win_score=b.get("win_score"), win_lse=b.get("win_lse"),
                              status=b.get("status"), workspace=b.get("ws_prefill"))
-    score = chunk_score if chunk_score is not None else chunk_score_from_lse(pre["win_lse"], out=b.get("chunk_score"))
-    kept = select_chunks(score, m, True, out=b.get("kept"))
+    if chunk_score is not None:
+        score, kept = chunk_score, select_chunks(chunk_score, m, True, out=b.get("kept"))
+    else:
+        score, kept = score_select_chunks(pre["win_lse"], m, True, score_out=b.get("chunk_score"), kept_out=b.get("kept"))
     idx = select_tokens(pre["win_score"], kept, L - w, k_keep, out=b.get("idx"))
     kc, vc, pos = gather_kv(pre["k_rot"], v, kept, idx, k_out=b.get("kc"), v_out=b.get("vc"), pos_out=b.get("pos"))
     # the window is the same in every chunk: take it from chunk 0 (views, no copy)
@@ -538,8 +554,7 @@ def hot_path_from_host(hq, hk, hv, *, w, rope_theta, m, k_keep, softmax_scale=0.
                                  out=b["o"][c0:c1], k_rot=b["k_rot"][c0:c1], win_score=b["win_score"][c0:c1],
                                  win_lse=b["win_lse"][c0:c1], status=b["status"], workspace=b.get("ws_prefill"))
         b["ws_prefill"] = pre["workspace"]
-    score = chunk_score_from_lse(b["win_lse"], out=b.get("chunk_score"))
-    kept = select_chunks(score, m, True, out=b.get("kept"))
+    score, kept = score_select_chunks(b["win_lse"], m, True, score_out=b.get("chunk_score"), kept_out=b.get("kept"))
     idx = select_tokens(b["win_score"], kept, L - w, k_keep, out=b.get("idx"))
     kc, vc, pos = gather_kv(b["k_rot"], v, kept, idx, k_out=b.get("kc"), v_out=b.get("vc"), pos_out=b.get("pos"))
     pa = parallel_attn(q[0:1, L - w:], kc.unsqueeze(0), vc.unsqueeze(0), b["k_rot"][0:1, L - w:], v[0:1, L - w:],

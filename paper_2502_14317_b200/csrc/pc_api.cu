@@ -236,6 +236,16 @@ int32_t pc_select_chunks(const float* chunk_score, int32_t C, int32_t m, int32_t
   return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------------------------ stand-in score + chunk top-m, one launch
+int32_t pc_score_select_chunks(const float* win_lse, int32_t C, int32_t Hq, int32_t w, int32_t m, int32_t lower_is_better,
+                               float* chunk_score, int32_t* kept, void* stream) {
+  if (!win_lse || !chunk_score || !kept || C < 1 || Hq < 1 || w < 1 || m < 1 || m > C) return PC_ERR_INVALID_ARG;
+  if (C > 1024) return PC_ERR_UNSUPPORTED;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  pc::launch_score_select_chunks(win_lse, C, Hq * w, m, lower_is_better, chunk_score, kept, static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? PC_OK : PC_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------------------------ token top-k
 int32_t pc_select_tokens(const float* win_score, const int32_t* kept, int32_t C, int32_t m, int32_t Hkv, int32_t L,
                          int32_t n_cand, int32_t k, int32_t* idx, void* stream) {

@@ -193,6 +193,12 @@ __device__ __forceinline__ void rope_row_smem(uint8_t* tile, int row, const doub
   }
 }
 
+// One arrival for a whole warp (an arrival per thread costs the barrier 32 serialised shared-memory operations).
+__device__ __forceinline__ void warp_arrive(uint64_t* bar) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
+
 // ------------------------------------------------------------------ softmax of one tile (thread = row)
 // Reads the 128 fp32 logits of this thread's row from TMEM, updates the running
 // (m, l), rescales the accumulator when the maximum moved by more than 2^LAZY_RESCALE,
@@ -261,7 +267,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_taddr, uint32_t o_taddr,
     if (q == 1) {                                                 // keys 0..63 of P are final: the issuer may start P V on them
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(p_half_bar);
+      warp_arrive(p_half_bar);
     }
   }
   float a0, a1, a2, a3;
@@ -324,11 +330,11 @@ struct Ctx {
 __device__ __forceinline__ void init_barriers(Misc& mi, int wait_kcycles) {
 #pragma unroll
   for (int b = 0; b < 2; ++b) {
-    mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 128); mbar_init(&mi.q_free[b], 1);
-    mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_half[b], 128); mbar_init(&mi.p_full[b], 128); mbar_init(&mi.o_full[b], 1);
-    mbar_init(&mi.acc_free[b], 128);
-    mbar_init(&mi.item_full[b], 1); mbar_init(&mi.item_empty[b], 258);
-    mbar_init(&mi.t_full[b], 2); mbar_init(&mi.t_free[b], 256);
+    mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 4); mbar_init(&mi.q_free[b], 1);        // groups arrive once per warp
+    mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_half[b], 4); mbar_init(&mi.p_full[b], 4); mbar_init(&mi.o_full[b], 1);
+    mbar_init(&mi.acc_free[b], 4);
+    mbar_init(&mi.item_full[b], 1); mbar_init(&mi.item_empty[b], 10);      // 8 softmax warps + 2 issuer threads
+    mbar_init(&mi.t_full[b], 2); mbar_init(&mi.t_free[b], 8);
     mbar_init(&mi.turn[b], 1);
   }
   for (int s = 0; s < NS; ++s) { mbar_init(&mi.kv_full[s], 1); mbar_init(&mi.kv_free[s], 2); }   // both issuers release a stage
@@ -353,12 +359,13 @@ __device__ __forceinline__ int producer_next_item(const Ctx& cx, Waits& wt, int*
   return item;
 }
 // consumers: read the next work item
-__device__ __forceinline__ int consumer_next_item(const Ctx& cx, Waits& wt) {
+// whole_warp: called by all 32 threads of a softmax warp (one arrival for the warp); else by a single issuer thread
+__device__ __forceinline__ int consumer_next_item(const Ctx& cx, Waits& wt, bool whole_warp) {
   Misc& mi = *cx.mi;
   const int slot = wt.item & 1;
   if (!mbar_wait(&mi.item_full[slot], full_par(wt.item >> 1), cx.abort_flag, cx.status, W_ITEM)) return ITEM_DONE;   // aborted: stop
   const int item = mi.item_slot[slot];
-  mbar_arrive(&mi.item_empty[slot]);
+  if (whole_warp) warp_arrive(&mi.item_empty[slot]); else mbar_arrive(&mi.item_empty[slot]);
   ++wt.item;
   return item;
 }
@@ -487,7 +494,7 @@ __device__ __forceinline__ void wg_flash_loop(const Ctx& cx, uint32_t& n_s, uint
     tc_fence_after_sync();
     softmax_tile<D>(tS, tO, vis(j), j == 0, scale_log2, m_used, l_run, &mi.p_half[b]);
     tc_fence_before_sync();
-    mbar_arrive(&mi.p_full[b]);
+    warp_arrive(&mi.p_full[b]);
   }
   mbar_wait(&mi.o_full[b], full_par(n_o), cx.abort_flag, cx.status, W_OFULL);
   ++n_o;
@@ -594,7 +601,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint32_t ring_u32 = smem_u32(cx.ring);
       const uint32_t q_u32 = smem_u32(cx.sQ[b]);
       while (true) {
-        const int item = consumer_next_item(cx, wt);
+        const int item = consumer_next_item(cx, wt, false);
         if (item == ITEM_DONE) break;
         const int group = item / sch.ipg, within = item % sch.ipg;
         const int hkv = group % prm.Hkv;
@@ -648,7 +655,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint8_t* const myQ = b ? cx.sQ[1] : cx.sQ[0];
     uint32_t n_s = 0, n_o = 0, n_t0 = 0, n_t1 = 0;            // barrier use counts of this group
     while (true) {
-      const int item = consumer_next_item(cx, wt);
+      const int item = consumer_next_item(cx, wt, true);
       if (item == ITEM_DONE) break;
       const int group = item / sch.ipg, within = item % sch.ipg;
       const int c = group / prm.Hkv, hkv = group % prm.Hkv;
@@ -685,7 +692,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
         tc_fence_before_sync();
-        mbar_arrive(&mi.acc_free[b]);
+        warp_arrive(&mi.acc_free[b]);
         const float lse2 = m_used + log2f(l_run);
         if (in_chunk) {
           if (prm.lse) prm.lse[((size_t)c * prm.Hq + h) * prm.L + token] = lse2 * 0.6931471805599453f;
@@ -737,7 +744,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               }
             }
             tc_fence_before_sync();
-            mbar_arrive(&mi.t_free[e]);
+            warp_arrive(&mi.t_free[e]);
             if (b == 1) mi.xch[e][r] = part;
             named_barrier_sync(3, 256);
             if (b == 0 && key < len) {
@@ -862,7 +869,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
     if (lane == 0) {
       const int b = warp - WARP_MMA;
       while (true) {
-        const int item = consumer_next_item(cx, wt);
+        const int item = consumer_next_item(cx, wt, false);
         if (item == ITEM_DONE) break;
         const Dec d = decode(item);
         const bool has_b = d.rows[b] > 0;
@@ -880,7 +887,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
     uint32_t n_q = 0, n_s = 0, n_o = 0;
     const int wi = r % prm.w;                                 // window index of this row (128 % w == 0)
     while (true) {
-      const int item = consumer_next_item(cx, wt);
+      const int item = consumer_next_item(cx, wt, true);
       if (item == ITEM_DONE) break;
       const Dec d = decode(item);
       const int rows_b = b ? d.rows[1] : d.rows[0];
@@ -889,7 +896,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
       ++n_q;
       if (r < rows_b) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)wi * (D / 2));
       fence_proxy_async_smem();
-      mbar_arrive(&mi.q_rot[b]);
+      warp_arrive(&mi.q_rot[b]);
       float m_used, l_run;
       wg_flash_loop<D>(cx, n_s, n_o, b, tS, tO, d.n, prm.scale_log2,
                        [&](int jj) {
@@ -939,7 +946,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
         if (valid) reinterpret_cast<float2*>(prm.part_ml)[prow] = make_float2(m_used, l_run);
       }
       tc_fence_before_sync();
-      mbar_arrive(&mi.acc_free[b]);
+      warp_arrive(&mi.acc_free[b]);
     }
   }
 

@@ -27,6 +27,9 @@ void launch_zero_chunk_tails(const int* chunk_len, int C, int L, int w, int Hq, 
 // ---- pc_select_gather.cu
 void launch_chunk_score(const float* win_lse, int C, int n_per_chunk, float* score, cudaStream_t st);
 void launch_select_chunks(const float* score, int C, int m, int lower_is_better, int* kept, cudaStream_t st);
+// stand-in chunk score (as launch_chunk_score, same bits) followed by the chunk top-m, in one launch for C <= 64
+void launch_score_select_chunks(const float* win_lse, int C, int n_per_chunk, int m, int lower_is_better, float* score,
+                                int* kept, cudaStream_t st);
 // calib: null, or host array {n_s, n_r, lam_s, lam_m, lam_r} (attention calibration, Eq. 8)
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
                                  int* idx, const float* calib, cudaStream_t st);

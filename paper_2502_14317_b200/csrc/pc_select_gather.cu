@@ -51,6 +51,61 @@ __global__ void select_chunks_kernel(const float* __restrict__ score, int C, int
   }
 }
 
+// Stand-in score and chunk top-m in ONE launch (C <= 64): four groups of 256 threads reduce the chunks' window
+// log-sum-exp in the order of chunk_score_kernel (same bits), then the block ranks them.
+__global__ void __launch_bounds__(1024) score_select_chunks_kernel(const float* __restrict__ win_lse, int n_per_chunk, int C,
+                                                                   int m, int lower_is_better, float* __restrict__ score,
+                                                                   int* __restrict__ kept) {
+  __shared__ double part[4][256];
+  __shared__ uint32_t key[64];
+  __shared__ int flag[64];
+  const int grp = threadIdx.x >> 8, t = threadIdx.x & 255;
+  for (int c0 = 0; c0 < C; c0 += 4) {                        // the barriers inside are reached by every thread
+    const int c = c0 + grp;
+    double acc = 0.0;
+    if (c < C)
+      for (int i = t; i < n_per_chunk; i += 256) acc += (double)win_lse[(size_t)c * n_per_chunk + i];
+    part[grp][t] = acc;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) {
+      if (t < s) part[grp][t] += part[grp][t + s];
+      __syncthreads();
+    }
+    if (t == 0 && c < C) {
+      const float sc = (float)(-part[grp][0] / (double)n_per_chunk);
+      score[c] = sc;
+      key[c] = rank_key(sc, lower_is_better != 0);
+    }
+    __syncthreads();
+  }
+  const int i = threadIdx.x;
+  int sel = 0;
+  if (i < C) {
+    const uint32_t mine = key[i];
+    int rank = 0;
+    for (int j = 0; j < C; ++j) rank += (key[j] > mine) || (key[j] == mine && j < i);
+    sel = rank < m;
+    flag[i] = sel;
+  }
+  __syncthreads();
+  if (sel) {
+    int pos = 0;
+    for (int j = 0; j < i; ++j) pos += flag[j];
+    kept[pos] = i;
+  }
+}
+
+void launch_score_select_chunks(const float* win_lse, int C, int n_per_chunk, int m, int lower_is_better, float* score,
+                                int* kept, cudaStream_t st) {
+  if (C <= 64) {
+    note_launch();
+    score_select_chunks_kernel<<<1, 1024, 0, st>>>(win_lse, n_per_chunk, C, m, lower_is_better, score, kept);
+  } else {
+    launch_chunk_score(win_lse, C, n_per_chunk, score, st);
+    launch_select_chunks(score, C, m, lower_is_better, kept, st);
+  }
+}
+
 void launch_select_chunks(const float* score, int C, int m, int lower_is_better, int* kept, cudaStream_t st) {
   note_launch();
   select_chunks_kernel<<<1, 1024, 0, st>>>(score, C, m, lower_is_better, kept);

@@ -134,3 +134,23 @@ def test_select_tokens_calibrated(C, m, L, w, k, Hkv, n_s, n_r, lams):
                                     lambda_s=inf, lambda_m=inf, lambda_r=inf)
     b = pc.select_tokens(torch.from_numpy(S).cuda(), torch.from_numpy(kept).cuda(), L - w, k)
     assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("C,Hq,w,m", [(16, 32, 64, 8), (4, 4, 16, 2), (64, 8, 24, 17), (7, 3, 5, 7), (100, 4, 8, 30)])
+def test_score_and_chunk_ranking_in_one_call(C, Hq, w, m):
+    """pc_score_select_chunks = pc_chunk_score_from_lse + pc_select_chunks, bit for bit (one launch up to 64 chunks,
+    two beyond), and the oracle's selection on that score."""
+    import paper_2502_14317_b200 as pc
+    rng = np.random.default_rng(C * 31 + w)
+    lse = rng.standard_normal((C, Hq, w)).astype(np.float32) * 3 + 7
+    if C > 4:
+        lse[3] = lse[1]                                          # a tie between two chunks
+    d = _dev(lse)
+    score_a = pc.chunk_score_from_lse(d)
+    kept_a = pc.select_chunks(score_a, m, True)
+    n0 = pc.launch_count()
+    score_b, kept_b = pc.score_select_chunks(d, m, True)
+    assert pc.launch_count() - n0 == (1 if C <= 64 else 2)
+    torch.cuda.synchronize()
+    assert torch.equal(score_a.view(torch.int32), score_b.view(torch.int32)) and torch.equal(kept_a, kept_b)
+    assert np.array_equal(kept_b.cpu().numpy(), orc.select_chunks(score_b.cpu().numpy(), m, True))
