@@ -222,7 +222,7 @@ PC_API int32_t pc_gather_kv(const void* k_src, const void* v_src, const int64_t*
  *
  * The chunks of a long input arrive in batches.  For every batch the caller runs
  * pc_chunk_prefill_attn, scores the chunks, runs pc_select_tokens over ALL chunks of the
- * batch (kept = 0..Cb-1), then
+ * batch (kept = 0..Cb-1) - or leaves that to pc_queue_select_gather below - then
  *   pc_queue_update  decides which of the m queued chunks and Cb new chunks stay: the m best
  *                    scores (lowest if lower_is_better != 0; ties go to the lower chunk id;
  *                    NaN ranks worst; empty slots rank below everything).  A chunk that stays
@@ -254,6 +254,19 @@ PC_API int32_t pc_queue_update(const float* chunk_score, int32_t Cb, int32_t chu
 PC_API int32_t pc_queue_gather(const void* k_src, const void* v_src, const int64_t* kv_stride,
                         const int32_t* slot_src, const int32_t* idx, int32_t m, int32_t Hkv, int32_t k, int32_t d,
                         void* q_k, void* q_v, int32_t* q_pos, void* stream);
+
+/* pc_select_tokens and pc_queue_gather in one launch, for the chunks that enter the queue only (a chunk
+ * that does not enter is dropped whole, so its tokens need no ranking): for every slot s with
+ * c = slot_src[s] >= 0 and every kv-head, the k best of win_score[c, hkv, 0..n_cand) are ranked as
+ * pc_select_tokens ranks them, their positions go to q_pos[hkv, s*k + t] and their rows of k_src / v_src
+ * to q_k / q_v[hkv, s*k + t, :]; the block that ranked a row copies it, the index list never travels
+ * through global memory.  Same results as the two calls.  win_score [Cb,Hkv,L] of the batch.
+ * PC_ERR_UNSUPPORTED if k > 10240 (use the two calls then).
+ */
+PC_API int32_t pc_queue_select_gather(const float* win_score, const void* k_src, const void* v_src,
+                               const int64_t* kv_stride, const int32_t* slot_src, int32_t m, int32_t Hkv,
+                               int32_t L, int32_t n_cand, int32_t k, int32_t d, void* q_k, void* q_v,
+                               int32_t* q_pos, void* stream);
 
 PC_API int32_t pc_queue_emit(const int32_t* q_chunk, int32_t m, int32_t Hkv, int32_t k, int32_t d, const void* q_k,
                       const void* q_v, const int32_t* q_pos, int32_t* kept_out, int32_t* slot_order, void* k_out,

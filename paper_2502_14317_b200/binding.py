@@ -76,6 +76,8 @@ def load_library():
     lib.pc_queue_gather.restype = c_int32
     lib.pc_queue_gather.argtypes = [c_void_p, c_void_p, POINTER(c_int64), c_void_p, c_void_p] + [c_int32] * 4 + \
         [c_void_p] * 4
+    lib.pc_queue_select_gather.restype = c_int32
+    lib.pc_queue_select_gather.argtypes = [c_void_p, c_void_p, c_void_p, POINTER(c_int64), c_void_p] + [c_int32] * 6 + [c_void_p] * 4
     lib.pc_queue_emit.restype = c_int32
     lib.pc_queue_emit.argtypes = [c_void_p] + [c_int32] * 4 + [c_void_p] * 9
     lib.pc_parallel_attn_workspace_bytes.restype = c_size_t
@@ -320,6 +322,22 @@ def queue_gather(state, k_src, v_src, idx):
            "pc_queue_gather")
 
 
+def queue_select_gather(state, win_score, k_src, v_src, n_cand):
+    """pc_queue_select_gather: rank the tokens of the chunks that entered the queue and move their kept rows into
+    their slots, one launch.  win_score [Cb,Hkv,L] fp32, k_src/v_src [Cb,L,Hkv,d] bf16 of the batch."""
+    lib = load_library()
+    _need_cuda(win_score, k_src, v_src)
+    Cb, L, Hkv, d = k_src.shape
+    if Hkv != state["Hkv"] or d != state["d"] or win_score.shape != (Cb, Hkv, L) or not win_score.is_contiguous():
+        raise PcError("win_score must be contiguous [Cb, Hkv, L]; Hkv and d must match the queue")
+    if k_src.stride() != v_src.stride() or k_src.stride(3) != 1:
+        raise PcError("k_src and v_src must share strides with a contiguous head dimension")
+    strides = (c_int64 * 3)(k_src.stride(0), k_src.stride(1), k_src.stride(2))
+    _check(lib.pc_queue_select_gather(_ptr(win_score), _ptr(k_src), _ptr(v_src), strides, _ptr(state["slot_src"]), state["m"],
+                                      Hkv, L, int(n_cand), state["k"], d, _ptr(state["q_k"]), _ptr(state["q_v"]),
+                                      _ptr(state["q_pos"]), _stream()), "pc_queue_select_gather")
+
+
 def queue_emit(state, k_out=None, v_out=None, pos_out=None, kept_out=None):
     """pc_queue_emit: the surviving chunks in ascending id order -> (kept [m], k_out, v_out [Hkv, m*k, d], pos [Hkv, m*k])."""
     lib = load_library()
@@ -437,8 +455,8 @@ def hot_path_streaming(q, k, v, *, w, rope_theta, m, k_keep, batch=None, softmax
                        buffers=None):
     """The whole path with the chunks taken one batch at a time through the online chunk queue.
 
-    Per batch: chunk-local attention, token eviction on EVERY chunk of the batch, queue update, and the
-    compressed caches of the chunks that entered the queue are copied into their slots; the batch's outputs
+    Per batch: chunk-local attention, queue update, then the chunks that entered the queue are ranked per kv-head
+    and their kept rows copied into their slots (one launch; a chunk that does not enter is dropped whole); the batch's outputs
     (attention output, rotated keys, window scores) live in buffers of batch size that the next batch
     overwrites, so device memory beyond the inputs is O(batch + m) chunks whatever C is.  After the last batch
     the queue is emitted in chunk order and the window attends over it.  Same results as :func:`hot_path`
@@ -489,10 +507,13 @@ def hot_path_streaming(q, k, v, *, w, rope_theta, m, k_keep, batch=None, softmax
         else:
             score = chunk_score_from_lse(pre["win_lse"], out=pb.get("score"))
             pb["score"] = score
-        idx = select_tokens(pre["win_score"], b["ids"][:n], L - w, k_keep, out=pb.get("idx"))
-        pb["idx"] = idx
         queue_update(qu, score, c0, True)
-        queue_gather(qu, pre["k_rot"], bv, idx)
+        if k_keep <= 10240:                                    # rank and compact the chunks that entered, one launch
+            queue_select_gather(qu, pre["win_score"], pre["k_rot"], bv, L - w)
+        else:
+            idx = select_tokens(pre["win_score"], b["ids"][:n], L - w, k_keep, out=pb.get("idx"))
+            pb["idx"] = idx
+            queue_gather(qu, pre["k_rot"], bv, idx)
         if k_win is None:                                      # the window is the same in every chunk: keep the first
             k_win = b.get("k_win")
             if k_win is None or k_win.shape != (1, w, Hkv, d):

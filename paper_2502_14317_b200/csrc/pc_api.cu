@@ -330,6 +330,23 @@ int32_t pc_queue_gather(const void* k_src, const void* v_src, const int64_t* kv_
   return PC_OK;
 }
 
+int32_t pc_queue_select_gather(const float* win_score, const void* k_src, const void* v_src, const int64_t* kv_stride,
+                               const int32_t* slot_src, int32_t m, int32_t Hkv, int32_t L, int32_t n_cand, int32_t k,
+                               int32_t d, void* q_k, void* q_v, int32_t* q_pos, void* stream) {
+  if (!win_score || !k_src || !v_src || !kv_stride || !slot_src || !q_k || !q_v || !q_pos) return PC_ERR_INVALID_ARG;
+  if (m < 1 || Hkv < 1 || L < 1 || n_cand < 1 || n_cand > L || k < 1) return PC_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return PC_ERR_UNSUPPORTED;
+  if (n_cand > 32768) return PC_ERR_UNSUPPORTED;
+  if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(q_k) || !aligned16(q_v)) return PC_ERR_INVALID_ARG;
+  const long long s[3] = {kv_stride[0], kv_stride[1], kv_stride[2]};
+  if (s[0] <= 0 || s[1] <= 0 || s[2] < d || s[0] % 8 || s[1] % 8 || s[2] % 8) return PC_ERR_INVALID_ARG;
+  if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
+  const cudaError_t e = pc::launch_select_gather_slots(win_score, slot_src, m, Hkv, L, n_cand, k, k_src, v_src, s, d, q_k,
+                                                       q_v, q_pos, static_cast<cudaStream_t>(stream));
+  if (e == cudaErrorNotSupported) return PC_ERR_UNSUPPORTED;     // k too large to stage: pc_select_tokens + pc_queue_gather
+  return e == cudaSuccess ? PC_OK : PC_ERR_CUDA;
+}
+
 int32_t pc_queue_emit(const int32_t* q_chunk, int32_t m, int32_t Hkv, int32_t k, int32_t d, const void* q_k,
                       const void* q_v, const int32_t* q_pos, int32_t* kept_out, int32_t* slot_order, void* k_out,
                       void* v_out, int32_t* pos_out, void* stream) {

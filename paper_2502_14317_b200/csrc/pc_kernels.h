@@ -33,6 +33,11 @@ void launch_score_select_chunks(const float* win_lse, int C, int n_per_chunk, in
 // calib: null, or host array {n_s, n_r, lam_s, lam_m, lam_r} (attention calibration, Eq. 8)
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
                                  int* idx, const float* calib, cudaStream_t st);
+// online chunk queue: rank the chunks that move into a slot (slot_src[s] >= 0) and copy their kept rows into the slot
+// storage, in one launch; cudaErrorNotSupported when k is too large for that (then rank and gather separately)
+cudaError_t launch_select_gather_slots(const float* win_score, const int* slot_src, int m, int Hkv, int L, int n_cand,
+                                       int k, const void* k_src, const void* v_src, const long long stride_elems[3],
+                                       int d, void* q_k, void* q_v, int* q_pos, cudaStream_t st);
 cudaError_t launch_gather_kv(const void* k_src, const void* v_src, const long long stride_elems[3], const int* kept,
                              const int* idx, int m, int Hkv, int k, int d, void* k_out, void* v_out, int* pos_out,
                              int sm_count, bool by_slot, cudaStream_t st);

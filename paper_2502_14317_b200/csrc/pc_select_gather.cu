@@ -184,14 +184,25 @@ __device__ __forceinline__ int sel_ordered_offsets(uint32_t x, int lane, int war
   return total;
 }
 
+// Copy of the kept rows by the block that ranked them (online chunk queue: a chunk that enters the queue is
+// ranked and compacted in one launch; chunks that do not enter are not ranked at all).
+struct SelGather {
+  const uint4* k_src; const uint4* v_src;                      // [Cb,L,Hkv,d] through strides in 16-byte units
+  long long s_chunk, s_tok, s_head;
+  uint4* k_out; uint4* v_out; int* pos_out;                    // slot storage [Hkv, m*k, d] x 2, [Hkv, m*k]
+  int lpr;                                                     // 16-byte pieces (= lanes) per row, d / 8
+};
+
 // STAGE: the kept positions are first put in order in shared memory (k words) and written out coalesced;
 // otherwise (k too large for that) they are stored straight to the index row.
 // SMALL: rows of at most 8192 candidates (256 threads), compiled for five CTAs per SM.
-template <bool CAL, bool STAGE, bool SMALL>
+// GATHER (with STAGE): kept[r] is the batch chunk that moves into queue slot r (-1: the slot keeps its contents and
+// the block returns); positions go to pos_out[hkv, r*k + t] and the rows k_src / v_src[kept[r], pos, hkv] to slot r.
+template <bool CAL, bool STAGE, bool SMALL, bool GATHER = false>
 __global__ void __launch_bounds__(SMALL ? 256 : SEL_MAX_THREADS, SMALL ? SEL_SMALL_CTAS : 1) select_tokens_kernel(const float* __restrict__ win_score,
                                                                         const int* __restrict__ kept, int Hkv, int L,
                                                                         int n_cand, int k, int* __restrict__ idx,
-                                                                        const SelCalib cal) {
+                                                                        const SelCalib cal, const SelGather ga = SelGather()) {
   extern __shared__ int sel_stage[];                           // STAGE: [min(k, n_cand)]
   __shared__ int s_part[2][32];                                // [round parity][warp]: undecided keys of the warp with the bit set
   __shared__ int s_tot[2][32];
@@ -199,14 +210,16 @@ __global__ void __launch_bounds__(SMALL ? 256 : SEL_MAX_THREADS, SMALL ? SEL_SMA
   const int row = blockIdx.x;                                  // r * Hkv + hkv
   const int r = row / Hkv, hk = row % Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  int* out = idx + (size_t)row * k;
+  const int n_slots = gridDim.x / Hkv;
+  int* out = GATHER ? ga.pos_out + ((size_t)hk * n_slots + r) * k : idx + (size_t)row * k;
+  if (GATHER && kept[r] < 0) return;                           // nothing moves into this slot
 
-  if (!CAL && k >= n_cand) {                                   // nothing to evict: identity, then -1 padding
+  if (!GATHER && !CAL && k >= n_cand) {                        // nothing to evict: identity, then -1 padding
     for (int j = tid; j < k; j += blockDim.x) out[j] = j < n_cand ? j : -1;
     return;
   }
   const int k_out = k;
-  if (k > n_cand) k = n_cand;                                  // calibrated: rank all candidates, pad the rest
+  if (k > n_cand) k = n_cand;                                  // rank all candidates, pad the rest
   const int c = kept[r];
   const float* src = win_score + ((size_t)c * Hkv + hk) * L;
 
@@ -351,6 +364,23 @@ __global__ void __launch_bounds__(SMALL ? 256 : SEL_MAX_THREADS, SMALL ? SEL_SMA
     }
     __syncthreads();
     for (int j = tid; j < k_out; j += blockDim.x) out[j] = j < n_emit ? sel_stage[j] : -1;
+    if (GATHER) {                                              // rows of the kept positions, lpr lanes per row, K and V together
+      const int rows_per_warp = 32 / ga.lpr, piece = lane % ga.lpr;
+      for (int j0 = warp * rows_per_warp; j0 < k_out; j0 += nwarps * rows_per_warp) {
+        const int j = j0 + lane / ga.lpr;
+        if (j >= k_out) continue;
+        const int pos = j < n_emit ? sel_stage[j] : -1;
+        uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
+        if (pos >= 0) {
+          const long long off = (long long)c * ga.s_chunk + (long long)pos * ga.s_tok + (long long)hk * ga.s_head + piece;
+          kv = __ldg(ga.k_src + off);
+          vv = __ldg(ga.v_src + off);
+        }
+        const size_t dst = (((size_t)hk * n_slots + r) * k_out + j) * ga.lpr + piece;
+        ga.k_out[dst] = kv;
+        ga.v_out[dst] = vv;
+      }
+    }
   } else {
 #pragma unroll
     for (int i = 0; i < SEL_KPT; ++i) {
@@ -389,6 +419,32 @@ cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m,
     if (stage) PC_SELECT(false, true); else PC_SELECT(false, false);
   }
 #undef PC_SELECT
+  return cudaGetLastError();
+}
+
+// Ranking and compaction of the chunks that enter the online queue, one launch.  Returns cudaErrorNotSupported when
+// the kept positions of a row do not fit the staging buffer (the caller then ranks and gathers in two launches).
+cudaError_t launch_select_gather_slots(const float* win_score, const int* slot_src, int m, int Hkv, int L, int n_cand,
+                                       int k, const void* k_src, const void* v_src, const long long stride_elems[3],
+                                       int d, void* q_k, void* q_v, int* q_pos, cudaStream_t st) {
+  int threads = (n_cand + SEL_SPAN - 1) / SEL_SPAN * 32;
+  if (threads < 32) threads = 32;
+  if (threads > SEL_MAX_THREADS) return cudaErrorInvalidValue;
+  const size_t stage_bytes = sizeof(int) * (size_t)(k < n_cand ? k : n_cand);
+  if (stage_bytes > 40 * 1024) return cudaErrorNotSupported;
+  const SelCalib cal{0, 0, 0, 0.f, 0.f, 0.f};
+  SelGather ga;
+  ga.k_src = (const uint4*)k_src; ga.v_src = (const uint4*)v_src;
+  ga.s_chunk = stride_elems[0] / 8; ga.s_tok = stride_elems[1] / 8; ga.s_head = stride_elems[2] / 8;
+  ga.k_out = (uint4*)q_k; ga.v_out = (uint4*)q_v; ga.pos_out = q_pos;
+  ga.lpr = d / 8;
+  note_launch();
+  if (threads <= 256)
+    select_tokens_kernel<false, true, true, true><<<m * Hkv, threads, stage_bytes, st>>>(win_score, slot_src, Hkv, L, n_cand, k,
+                                                                                        nullptr, cal, ga);
+  else
+    select_tokens_kernel<false, true, false, true><<<m * Hkv, threads, stage_bytes, st>>>(win_score, slot_src, Hkv, L, n_cand, k,
+                                                                                         nullptr, cal, ga);
   return cudaGetLastError();
 }
 

@@ -200,3 +200,39 @@ def test_streaming_with_a_shorter_last_chunk(cfg0_inputs):
         check_attention_output(to_f64(got["fg"]), Fg, "Fg (ragged)")
     if forced is not None:
         assert 3 in kept_o.tolist()
+
+
+@pytest.mark.parametrize("Cb,L,w,Hkv,d,k,m", [(4, 256, 16, 2, 64, 64, 3), (3, 1100, 64, 2, 128, 300, 5), (2, 300, 24, 3, 128, 500, 2)])
+def test_rank_and_compact_in_one_launch_equals_the_two_calls(Cb, L, w, Hkv, d, k, m):
+    """pc_queue_select_gather = pc_select_tokens on the batch + pc_queue_gather, bit for bit: positions, keys and
+    values of the slots that take a chunk; slots that keep their contents are not touched.  (k above the number of
+    candidates in the last case: the tail of a slot is padded with position -1 and zero rows.)"""
+    import paper_2502_14317_b200 as pc
+    rng = np.random.default_rng(Cb * 100 + k)
+    score = torch.from_numpy(rng.random((Cb, Hkv, L)).astype(np.float32)).cuda()
+    ksrc = torch.from_numpy(rng.integers(0, 2 ** 15, size=(Cb, L, Hkv, d)).astype(np.int16)).cuda().view(torch.bfloat16)
+    vsrc = torch.from_numpy(rng.integers(0, 2 ** 15, size=(Cb, L, Hkv, d)).astype(np.int16)).cuda().view(torch.bfloat16)
+    slot_src = torch.full((m,), -1, dtype=torch.int32, device="cuda")
+    slot_src[0] = Cb - 1
+    if m > 2:
+        slot_src[2] = 0
+    states = []
+    for fused in (False, True):
+        st = pc.queue_init(m, Hkv, k, d, "cuda")
+        for key in ("q_k", "q_v"):
+            st[key].view(torch.int16).fill_(0x1234)                   # untouched slots must keep this
+        st["q_pos"].fill_(-7)
+        st["slot_src"].copy_(slot_src)
+        if fused:
+            n0 = pc.launch_count()
+            pc.queue_select_gather(st, score, ksrc, vsrc, L - w)
+            assert pc.launch_count() - n0 == 1
+        else:
+            idx = pc.select_tokens(score, torch.arange(Cb, dtype=torch.int32, device="cuda"), L - w, k)
+            pc.queue_gather(st, ksrc, vsrc, idx)
+        torch.cuda.synchronize()
+        states.append(st)
+    for key in ("q_k", "q_v"):
+        assert torch.equal(states[0][key].view(torch.int16), states[1][key].view(torch.int16)), key
+    assert torch.equal(states[0]["q_pos"], states[1]["q_pos"])
+    assert int((states[1]["q_pos"][:, k:2 * k] == -7).all()) == 1     # slot 1 keeps its contents
