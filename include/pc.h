@@ -319,8 +319,12 @@ PC_API int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, i
  *     (different streams, or different host threads on different streams) race on the
  *     array: serialise them on one stream or with events;
  *   - the first call on each device looks up the array's device address (a host-side
- *     query, no allocation, no launch).  Make that first call outside of any stream
+ *     query, no allocation call, no launch; where the CUDA runtime loads modules lazily this
+ *     is also when the driver binds the array's memory on that device).  Make that first call outside of any stream
  *     capture; later calls on that device skip the query.
+ *     The address is remembered per device ordinal for the life of the process: after a
+ *     cudaDeviceReset, or under a context other than the device's primary one, it is stale
+ *     and this entry point must not be used.
  * The call itself never calls cudaMalloc, cudaFree or any allocating routine.
  * Arguments, layouts, status word and return values otherwise as for pc_parallel_attn.
  */

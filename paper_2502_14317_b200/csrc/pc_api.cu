@@ -268,8 +268,8 @@ int32_t pc_select_tokens_calibrated(const float* win_score, const int32_t* kept,
   if (n_s < 0 || n_r < 0 || lambda_s != lambda_s || lambda_m != lambda_m || lambda_r != lambda_r) return PC_ERR_INVALID_ARG;
   if (n_cand > 32768) return PC_ERR_UNSUPPORTED;
   if (device_info().ok != 1) return PC_ERR_UNSUPPORTED;
-  const float calib[5] = {(float)n_s, (float)n_r, lambda_s, lambda_m, lambda_r};
-  if (pc::launch_select_tokens(win_score, kept, m, Hkv, L, n_cand, k, idx, calib, static_cast<cudaStream_t>(stream)) !=
+  const pc::SelCalibArgs calib{n_s, n_r, lambda_s, lambda_m, lambda_r};
+  if (pc::launch_select_tokens(win_score, kept, m, Hkv, L, n_cand, k, idx, &calib, static_cast<cudaStream_t>(stream)) !=
       cudaSuccess)
     return PC_ERR_CUDA;
   return PC_OK;

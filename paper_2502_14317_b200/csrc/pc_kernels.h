@@ -30,9 +30,13 @@ void launch_select_chunks(const float* score, int C, int m, int lower_is_better,
 // stand-in chunk score (as launch_chunk_score, same bits) followed by the chunk top-m, in one launch for C <= 64
 void launch_score_select_chunks(const float* win_lse, int C, int n_per_chunk, int m, int lower_is_better, float* score,
                                 int* kept, cudaStream_t st);
-// calib: null, or host array {n_s, n_r, lam_s, lam_m, lam_r} (attention calibration, Eq. 8)
+// attention calibration (Eq. 8): sizes of the sink and recency regions and the three thresholds; null = off
+struct SelCalibArgs {
+  int n_s, n_r;
+  float lam_s, lam_m, lam_r;
+};
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
-                                 int* idx, const float* calib, cudaStream_t st);
+                                 int* idx, const SelCalibArgs* calib, cudaStream_t st);
 // online chunk queue: rank the chunks that move into a slot (slot_src[s] >= 0) and copy their kept rows into the slot
 // storage, in one launch; cudaErrorNotSupported when k is too large for that (then rank and gather separately)
 cudaError_t launch_select_gather_slots(const float* win_score, const int* slot_src, int m, int Hkv, int L, int n_cand,

@@ -393,12 +393,13 @@ __global__ void __launch_bounds__(SMALL ? 256 : SEL_MAX_THREADS, SMALL ? SEL_SMA
 }
 
 cudaError_t launch_select_tokens(const float* win_score, const int* kept, int m, int Hkv, int L, int n_cand, int k,
-                                 int* idx, const float* calib /* null or {n_s, n_r, lam_s, lam_m, lam_r} */,
-                                 cudaStream_t st) {
+                                 int* idx, const SelCalibArgs* calib, cudaStream_t st) {
   int threads = (n_cand + SEL_SPAN - 1) / SEL_SPAN * 32;
   if (threads < 32) threads = 32;
   if (threads > SEL_MAX_THREADS) return cudaErrorInvalidValue;
-  const SelCalib cal = calib ? SelCalib{1, (int)calib[0], (int)calib[1], calib[2], calib[3], calib[4]}
+  // region sizes beyond the row mean "the whole row": clamp them on the host (they are compared with positions)
+  const SelCalib cal = calib ? SelCalib{1, calib->n_s < n_cand ? calib->n_s : n_cand, calib->n_r < n_cand ? calib->n_r : n_cand,
+                                        calib->lam_s, calib->lam_m, calib->lam_r}
                              : SelCalib{0, 0, 0, 0.f, 0.f, 0.f};
   const size_t stage_bytes = sizeof(int) * (size_t)(k < n_cand ? k : n_cand);
   const bool stage = stage_bytes <= 40 * 1024;                 // within the default dynamic shared-memory limit

@@ -21,24 +21,31 @@ def to_f64(t: torch.Tensor) -> np.ndarray:
 def check_attention_output(got_f64: np.ndarray, ref: np.ndarray, what: str = "O"):
     """Tolerance of the attention outputs: max-abs 1e-2, max-rel 2e-2.
 
-    Pure relative error is meaningless near zero and the bf16 output grid alone exceeds
-    1e-2 absolute for |x| > 4, so the element-wise gate is |d| <= 1e-2 + 2e-2 |ref|; the
-    two raw maxima are checked on the ranges where each is meaningful.  The tensor-core path
-    rounds the probabilities to bf16 (unit round-off 2^-9), which bounds the error of an output
-    by 2^-9 * sum_j A_ij |v_j| <= 2^-9 * max|v| (about 1e-2 for |v| up to 5); a relative bound of
-    2e-2 therefore follows from the arithmetic only where |ref| >= 2^-9 * max|v| / 2e-2 ~ 0.5.
-    """
+    Pure relative error is meaningless near zero and the bf16 output grid alone exceeds 1e-2 absolute for
+    |x| > 4, so the element-wise gate is |d| <= 1e-2 + 2e-2 |ref|, and the two raw maxima are checked on the
+    ranges where each is meaningful: max-abs <= 1e-2 where |ref| < 2 and <= 1.6e-2 where |ref| < 4 (half a bf16
+    step there is 3.9e-3 / 7.8e-3, the rest is the rounding of the probabilities); max-rel <= 2e-2 where
+    |ref| >= 0.5.  The tensor-core path rounds the probabilities to bf16 (unit round-off 2^-9), which bounds the
+    error of an output by 2^-9 * sum_j A_ij |v_j| <= 2^-9 * max|v| (about 1e-2 for |v| up to 5); a relative bound
+    of 2e-2 therefore follows from the arithmetic only where |ref| >= 2^-9 * max|v| / 2e-2 ~ 0.5.
+    Prints the two raw maxima with the |ref| at which they occur; returns the max-abs error."""
     d = np.abs(got_f64 - ref)
+    a = np.abs(ref)
     assert np.all(np.isfinite(got_f64)), f"{what}: non-finite values"
-    bad = d > 1e-2 + 2e-2 * np.abs(ref)
+    i_abs = int(np.argmax(d))
+    rel = d / np.maximum(a, 1e-30)
+    rel_dom = np.where(a >= 0.5, rel, 0.0)
+    i_rel = int(np.argmax(rel_dom))
+    print(f"{what}: max-abs {d.flat[i_abs]:.3e} at |ref| = {a.flat[i_abs]:.3f}; "
+          f"max-rel (|ref| >= 0.5) {rel_dom.flat[i_rel]:.3e} at |ref| = {a.flat[i_rel]:.3f}; {d.size} elements")
+    bad = d > 1e-2 + 2e-2 * a
     assert not bad.any(), f"{what}: {bad.sum()} elements outside 1e-2 + 2e-2|ref|, worst {d.max():.4e}"
-    small = np.abs(ref) <= 1.0
-    if small.any():
-        assert d[small].max() <= 1e-2, f"{what}: max-abs {d[small].max():.4e} on |ref| <= 1"
-    big = np.abs(ref) >= 0.5
-    if big.any():
-        rel = (d[big] / np.abs(ref[big])).max()
-        assert rel <= 2e-2, f"{what}: max-rel {rel:.4e} on |ref| >= 0.5"
+    for lim, cap in ((2.0, 1e-2), (4.0, 1.6e-2)):
+        band = a < lim
+        if band.any():
+            assert d[band].max() <= cap, f"{what}: max-abs {d[band].max():.4e} on |ref| < {lim}"
+    if (a >= 0.5).any():
+        assert rel_dom.max() <= 2e-2, f"{what}: max-rel {rel_dom.max():.4e} on |ref| >= 0.5"
     return float(d.max())
 
 

@@ -114,6 +114,8 @@ def test_keep_all_gather_is_a_reshape():
     (1, 1, 200, 8, 50, 1, 150, 150, (0.2, 0.3, 0.4)),           # overlapping regions: the sink region wins
     (2, 2, 400, 8, 30, 2, 100, 100, (0.0, 0.0, 0.0)),           # everything above the thresholds: all -1
     (1, 1, 16000, 64, 11000, 2, 100, 100, (0.9, 0.95, 0.9)),    # k too large for the staged output
+    (2, 2, 500, 12, 80, 2, 10 ** 6, 7, (0.7, 0.2, 0.3)),         # sink region larger than the row: it is the whole row
+    (1, 1, 300, 8, 40, 2, 3, 2 ** 31 - 1, (0.5, 0.2, 0.6)),      # recency region 'everything' (largest int32)
 ])
 def test_select_tokens_calibrated(C, m, L, w, k, Hkv, n_s, n_r, lams):
     import paper_2502_14317_b200 as pc
