@@ -330,6 +330,7 @@ def run_gpu(args, cfg):
 
     stage_ms = {name: statistics.mean(ev[s][a].elapsed_time(ev[s][b]) for s in range(args.steps))
                 for name, a, b in (("prefill_attn", 0, 1), ("score_select", 1, 2), ("gather", 2, 3), ("parallel_attn", 3, 4))}
+    prefill_ms_per_step = [ev[s][0].elapsed_time(ev[s][1]) for s in range(args.steps)]
 
     # ---- launch floor of the ranking stage: two launches that do (next to) nothing, timed like the stage
     tiny_lse = torch.zeros((1, 1, 1), dtype=torch.float32, device=dev)
@@ -408,6 +409,12 @@ def run_gpu(args, cfg):
                          "peak_source": peak_note,
                          "flop_per_clk_per_sm": (ach_tflops * 1e12 / (sm_mhz * 1e6 * sm_count)) if sm_mhz else None,
                          "algorithmic_flops_per_launch": flops, "ms_per_launch": stage_ms["prefill_attn"],
+                         "ms_per_launch_fastest": min(prefill_ms_per_step),
+                         "tflops_fastest_launch": flops / (min(prefill_ms_per_step) * 1e-3) / 1e12,
+                         "ms_per_launch_by_step": [round(x, 3) for x in prefill_ms_per_step],
+                         "power_note": "back-to-back launches run into the board power cap after roughly 50 ms (sw_power_cap): the "
+                                       "launch time then rises by about a tenth; ms_per_launch is the mean over the timed steps, "
+                                       "ms_per_launch_fastest the launch least affected",
                          "traffic": traffic, "traffic_note": traffic_note},
             "stages": {
                 "prefill_attn": {"ms": stage_ms["prefill_attn"], "tflops": ach_tflops},

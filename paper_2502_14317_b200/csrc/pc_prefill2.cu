@@ -723,22 +723,6 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               const int g = g_base + ih;
               if (g >= sch.G) break;                         // filler head
               const float* lse_head = mi.lse2 + g * prm.w;
-              if ((prm.w & 31) == 0) {                       // no pad columns, 32 at a time: one wait per 32 exponentials
-                for (int col = 0; col < prm.w; col += 32) {
-                  uint32_t sv[32];
-                  tmem_ld32(tT + ih * prm.w + col, sv);
-                  tmem_wait_ld();
-                  float p4[4] = {0.0f, 0.0f, 0.0f, 0.0f};      // fixed order: deterministic
-#pragma unroll
-                  for (int i = 0; i < 32; ++i) {
-                    float pv = fast_exp2(fmaf(__uint_as_float(sv[i]), scale_log2, -lse_head[col + i]));
-                    if (need_mask && key > w0 + col + i) pv = 0.0f;
-                    p4[i & 3] += pv;
-                  }
-                  part += (p4[0] + p4[1]) + (p4[2] + p4[3]);
-                }
-                continue;
-              }
               for (int col = 0; col < sch.wp; col += 8) {
                 uint32_t sv[8];
                 tmem_ld8(tT + ih * sch.wp + col, sv);
