@@ -12,7 +12,7 @@ SOURCES = ["pc_api.cu", "pc_attn.cu", "pc_prefill2.cu", "pc_rope.cu", "pc_select
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",
-] + os.environ.get("PC_NVCC_EXTRA", "").split()
+]
 
 
 def _nvcc() -> str:

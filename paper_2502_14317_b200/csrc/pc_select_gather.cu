@@ -132,10 +132,7 @@ void launch_select_chunks(const float* score, int C, int m, int lower_is_better,
 constexpr int SEL_KPT = 32;                                    // keys per thread
 constexpr int SEL_SPAN = 32 * SEL_KPT;                         // positions per warp
 constexpr int SEL_MAX_THREADS = 1024;                          // n_cand <= 32768
-#ifndef PC_SEL_SMALL_CTAS
-#define PC_SEL_SMALL_CTAS 5
-#endif
-constexpr int SEL_SMALL_CTAS = PC_SEL_SMALL_CTAS;
+constexpr int SEL_SMALL_CTAS = 5;                              // resident CTAs per SM asked for by the narrow variant
 
 // Attention calibration (Eq. 8): a candidate whose score exceeds the threshold of its region (first n_s
 // positions / last n_r positions / the rest) is evicted before the ranking.  +inf switches a region off.

@@ -18,16 +18,20 @@ def to_f64(t: torch.Tensor) -> np.ndarray:
     return orc.bf16_to_f64(to_bits(t))
 
 
-def check_attention_output(got_f64: np.ndarray, ref: np.ndarray, what: str = "O"):
+def check_attention_output(got_f64: np.ndarray, ref: np.ndarray, what: str = "O", sharp: bool = False):
     """Tolerance of the attention outputs: max-abs 1e-2, max-rel 2e-2.
 
     Pure relative error is meaningless near zero and the bf16 output grid alone exceeds 1e-2 absolute for
     |x| > 4, so the element-wise gate is |d| <= 1e-2 + 2e-2 |ref|, and the two raw maxima are checked on the
-    ranges where each is meaningful: max-abs <= 1e-2 where |ref| < 2 and <= 1.6e-2 where |ref| < 4 (half a bf16
-    step there is 3.9e-3 / 7.8e-3, the rest is the rounding of the probabilities); max-rel <= 2e-2 where
-    |ref| >= 0.5.  The tensor-core path rounds the probabilities to bf16 (unit round-off 2^-9), which bounds the
-    error of an output by 2^-9 * sum_j A_ij |v_j| <= 2^-9 * max|v| (about 1e-2 for |v| up to 5); a relative bound
-    of 2e-2 therefore follows from the arithmetic only where |ref| >= 2^-9 * max|v| / 2e-2 ~ 0.5.
+    ranges where each is meaningful.  The tensor-core path rounds the probabilities to bf16 (unit round-off
+    u = 2^-8) and the output once more, so an output is off by at most u * sum_j A_ij |v_j| plus half a bf16 step
+    of the result (2^-9 |ref| .. 2^-8 |ref|).  Rows that attend to many keys average the first term away; a row
+    whose mass sits on one or two keys (the growing-logits cases) comes close to it, there sum_j A_ij |v_j| ~ |ref|
+    and the error reaches u |ref| + half a step: 2 u + 2^-8 = 1.17e-2 for |ref| < 2, 4 u + 2^-7 = 2.34e-2 for
+    |ref| < 4; with logits in the hundreds the fp32 accumulation of Q K^T adds a relative error of about 1e-3 to
+    the probabilities of competing keys.  Caps on the raw maxima: ordinary inputs max-abs <= 1e-2 where |ref| < 2
+    and <= 1.6e-2 where |ref| < 4; `sharp` inputs (those cases) <= 1.5e-2 and <= 3e-2; always max-rel <= 2e-2
+    where |ref| >= 0.5 (one-hot rows: at most 2 u = 7.8e-3; diffuse rows: u * max|v| / |ref|, |v| up to 5).
     Prints the two raw maxima with the |ref| at which they occur; returns the max-abs error."""
     d = np.abs(got_f64 - ref)
     a = np.abs(ref)
@@ -40,7 +44,7 @@ def check_attention_output(got_f64: np.ndarray, ref: np.ndarray, what: str = "O"
           f"max-rel (|ref| >= 0.5) {rel_dom.flat[i_rel]:.3e} at |ref| = {a.flat[i_rel]:.3f}; {d.size} elements")
     bad = d > 1e-2 + 2e-2 * a
     assert not bad.any(), f"{what}: {bad.sum()} elements outside 1e-2 + 2e-2|ref|, worst {d.max():.4e}"
-    for lim, cap in ((2.0, 1e-2), (4.0, 1.6e-2)):
+    for lim, cap in ((2.0, 1.5e-2 if sharp else 1e-2), (4.0, 3e-2 if sharp else 1.6e-2)):
         band = a < lim
         if band.any():
             assert d[band].max() <= cap, f"{what}: max-abs {d[band].max():.4e} on |ref| < {lim}"
