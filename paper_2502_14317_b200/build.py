@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libpc.so")
-SOURCES = ["pc_api.cu", "pc_attn.cu", "pc_prefill2.cu", "pc_rope.cu", "pc_select_gather.cu", "pc_queue.cu", "pc_static_scratch.cu"]
+SOURCES = ["pc_api.cu", "pc_attn.cu", "pc_prefill2.cu", "pc_parallel2.cu", "pc_rope.cu", "pc_select_gather.cu", "pc_queue.cu", "pc_static_scratch.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",

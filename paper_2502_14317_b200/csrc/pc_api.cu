@@ -370,11 +370,16 @@ namespace {
 
 struct ParallelPlan {
   int Gs, n_rg, n_cache_tiles, n_split, tiles_per_split;
-  size_t off_counter, off_table, off_ml, off_o, total;
+  bool pair;                       // CTA-pair kernel: 256-row groups, no key split
+  int hpc, n_rg_pair;              // pair kernel: q-heads per CTA, 256-row groups per kv-head
+  size_t off_counter, off_table, off_table_hi, off_table_lo, off_qrot, off_ml, off_o, total;
 };
 
 // Split the keys so that the persistent grid has a few items per SM; every split keeps at
 // least two cache tiles.  The plan depends only on the sizes and the SM count.
+// Head size 128 with whole 256-row groups per (sequence, kv-head) runs on CTA pairs, one group per pair and
+// item, without a key split, when the groups fill the pairs' rounds to three quarters or more (the pair kernel is
+// about a third faster per tile, a partly filled last round costs it that advantage).
 ParallelPlan parallel_plan(int B, int w, int Hq, int Hkv, int d, int Nk, int sm_count) {
   ParallelPlan p;
   const int G = Hq / Hkv;
@@ -382,17 +387,35 @@ ParallelPlan parallel_plan(int B, int w, int Hq, int Hkv, int d, int Nk, int sm_
   p.n_rg = (G + p.Gs - 1) / p.Gs;
   p.n_cache_tiles = (Nk + 127) / 128;
   const long long base = (long long)B * Hkv * p.n_rg;
+  p.pair = false;
+  p.hpc = 0; p.n_rg_pair = 0;
+  if (d == 128 && w >= 8 && (G * w) % 256 == 0 && sm_count >= 2) {
+    const long long pairs = sm_count / 2, groups = (long long)B * Hkv * (G * w / 256);
+    const long long rounds = (groups + pairs - 1) / pairs;
+    if (4 * groups >= 3 * rounds * pairs) {
+      p.pair = true;
+      p.hpc = 128 / w;
+      p.n_rg_pair = G * w / 256;
+    }
+  }
   long long want = (4LL * sm_count + base - 1) / base;
   long long cap = p.n_cache_tiles / 2;
   if (cap < 1) cap = 1;
   if (want > cap) want = cap;
   if (want < 1) want = 1;
+  if (p.pair) want = 1;
   p.tiles_per_split = (int)((p.n_cache_tiles + want - 1) / want);
   if (p.tiles_per_split < 1) p.tiles_per_split = 1;
   p.n_split = p.n_cache_tiles > 0 ? (p.n_cache_tiles + p.tiles_per_split - 1) / p.tiles_per_split : 1;
   size_t off = 0;
   p.off_counter = off; off += ALIGN;
   p.off_table = off; off += align_up((size_t)w * (d / 2) * sizeof(double2));
+  p.off_table_hi = off;
+  if (p.pair) off += align_up((size_t)w * (d / 4) * sizeof(float4));
+  p.off_table_lo = off;
+  if (p.pair) off += align_up((size_t)w * (d / 4) * sizeof(float4));
+  p.off_qrot = off;
+  if (p.pair) off += align_up((size_t)B * w * Hq * d * 2);
   p.off_ml = off;
   if (p.n_split > 1) off += align_up((size_t)B * Hq * p.n_split * w * 2 * sizeof(float));
   p.off_o = off;
@@ -444,7 +467,6 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   int* counter = reinterpret_cast<int*>(ws + plan.off_counter);
   double2* table = reinterpret_cast<double2*>(ws + plan.off_table);
 
-  CUtensorMap maps[5];
   const uint64_t ud = (uint64_t)d;
   const uint64_t qw_dims[4] = {ud, (uint64_t)Hq, (uint64_t)w, (uint64_t)B};
   const uint64_t qw_str[3] = {ud, (uint64_t)Hq * ud, (uint64_t)w * Hq * ud};
@@ -455,6 +477,38 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   const uint32_t box_qw[4] = {64, 1, (uint32_t)w, 1};
   const uint32_t box_kc[4] = {64, 128, 1, 1};
   const uint32_t box_kw[4] = {64, 1, 128, 1};
+
+  if (plan.pair) {
+    // rotated queries first (the same pass that serves the chunk-local kernel), then the pair kernel
+    float4* table_hi = reinterpret_cast<float4*>(ws + plan.off_table_hi);
+    float4* table_lo = reinterpret_cast<float4*>(ws + plan.off_table_lo);
+    void* q_rot = ws + plan.off_qrot;
+    pc::launch_rope_table(table, table_hi, table_lo, w, d, (double)rope_theta, q_pos0, st);
+    const long long q_stride[3] = {(long long)w * Hq * d, (long long)Hq * d, (long long)d};
+    pc::launch_rope_rows(q_win, q_stride, q_rot, table, table_hi, table_lo, B, w, Hq, d, st);
+    CUtensorMap pm[6];
+    const uint32_t box_kch[4] = {64, 64, 1, 1};
+    const uint32_t box_kwh[4] = {64, 1, 64, 1};
+    if (!pc::make_tmap_bf16_4d(&pm[0], q_rot, qw_dims, qw_str, box_qw) ||
+        !pc::make_tmap_bf16_4d(&pm[1], out, qw_dims, qw_str, box_qw) ||
+        !pc::make_tmap_bf16_4d(&pm[2], k_cache, kc_dims, kc_str, box_kch) ||
+        !pc::make_tmap_bf16_4d(&pm[3], v_cache, kc_dims, kc_str, box_kc) ||
+        !pc::make_tmap_bf16_4d(&pm[4], k_win, kw_dims, kw_str, box_kwh) ||
+        !pc::make_tmap_bf16_4d(&pm[5], v_win, kw_dims, kw_str, box_kw))
+      return PC_ERR_CUDA;
+    pc::ParallelPairParams pp;
+    pp.B = B; pp.w = w; pp.Hq = Hq; pp.Hkv = Hkv; pp.Nk = Nk;
+    pp.hpc = plan.hpc; pp.n_rg = plan.n_rg_pair;
+    const double scale = softmax_scale > 0.0f ? (double)softmax_scale : 1.0 / std::sqrt((double)d);
+    pp.scale_log2 = (float)(scale * 1.4426950408889634);
+    pp.lse_out = lse_out;
+    pp.status = status_word;
+    pp.wait_kcycles = pc::g_wait_kcycles.load();
+    if (pc::launch_parallel_pair(pm, pp, dev.sm_count, st) != cudaSuccess) return PC_ERR_CUDA;
+    return PC_OK;
+  }
+
+  CUtensorMap maps[5];
   if (!pc::make_tmap_bf16_4d(&maps[0], q_win, qw_dims, qw_str, box_qw) ||
       !pc::make_tmap_bf16_4d(&maps[1], k_cache, kc_dims, kc_str, box_kc) ||
       !pc::make_tmap_bf16_4d(&maps[2], v_cache, kc_dims, kc_str, box_kc) ||

@@ -44,4 +44,19 @@ struct ParallelParams {
 // maps: q_win (w-row box), k_cache, v_cache (128-key box), k_win, v_win (128-row box over w tokens)
 cudaError_t launch_parallel_attn(const CUtensorMap* maps, const ParallelParams& prm, int d, int grid, cudaStream_t st);
 
+// Parallel attention on CTA pairs (head size 128, G * w a multiple of 256, no key split): every pair takes the
+// windows of 2 * hpc q-heads of one kv-head (hpc * w = 128 rows per CTA) over the whole cache.
+struct ParallelPairParams {
+  int B, w, Hq, Hkv, Nk;
+  int hpc, n_rg;                 // q-heads per CTA, 256-row groups per kv-head
+  float scale_log2;
+  float* lse_out;                // [B,Hq,w] or null
+  int* status;
+  int wait_kcycles;              // limit of every device-side wait, in units of 1024 cycles
+};
+
+// maps: rotated q_win (box 64 x 1 head x w tokens), out (same box), k_cache (64 x 64 keys), v_cache (64 x 128 keys),
+// k_win (64 x 1 head x 64 tokens), v_win (64 x 1 head x 128 tokens)
+cudaError_t launch_parallel_pair(const CUtensorMap* maps, const ParallelPairParams& prm, int sm_count, cudaStream_t st);
+
 }  // namespace pc

@@ -36,19 +36,21 @@ void launch_rope_table(double2* tab, float4* tab_hi, float4* tab_lo, int n_pos, 
   rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, tab_hi, tab_lo, n_pos, d / 2, theta, pos0);
 }
 
-// y[c,p,h,:] = bf16( RoPE(x[c,p,h,:], position p) ).  One thread owns 8 consecutive pairs (t .. t+7) of one
-// position and walks all heads and a slice of the chunks, so its table entries are read once and stay in
-// registers.  A warp covers 32 / (d/16) positions: every 16-byte access of a warp falls into fully used
-// 128-byte segments.
+// y[c,p,h,:] = bf16( RoPE(x[c,p,h,:], position p) ).  One warp owns one position: a lane holds 8 consecutive
+// pairs (t .. t+7) and takes every (32 / (d/16))-th head, so one pass of the warp reads and writes a contiguous
+// piece of the token's row (1 KB for d = 128), and a block of 8 warps streams 8 adjacent rows: the DRAM pages
+// are walked front to back, as a copy would.  The table entries of (position, pairs) stay in registers across
+// the heads and across the chunks of the block's slice.
 __global__ void __launch_bounds__(256, 4) rope_rows_kernel(const uint16_t* __restrict__ x, long long s_chunk, long long s_tok,
                                                            long long s_head, uint16_t* __restrict__ y,
                                                            const float4* __restrict__ tab_hi, const float4* __restrict__ tab_lo,
                                                            const double2* __restrict__ tab, int C, int L, int H, int d) {
   const int half = d / 2;
-  const int groups = half / 8;                              // 16-byte groups per half row
-  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (gid >= (long long)L * groups) return;
-  const int p = (int)(gid / groups), g = (int)(gid % groups);
+  const int groups = half / 8;                              // 16-byte groups per half row (4 or 8)
+  const int lane = threadIdx.x & 31;
+  const int p = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (p >= L) return;
+  const int g = lane % groups, h_first = lane / groups, h_step = 32 / groups;
   const size_t e0 = (size_t)p * half + g * 8;               // first pair of this thread in the tables
   float4 hi[4];
 #pragma unroll
@@ -57,7 +59,7 @@ __global__ void __launch_bounds__(256, 4) rope_rows_kernel(const uint16_t* __res
     const uint16_t* src_c = x + (long long)c * s_chunk + (long long)p * s_tok + g * 8;
     uint16_t* dst_c = y + ((size_t)c * L + p) * H * d + g * 8;
 #pragma unroll 1
-    for (int h = 0; h < H; ++h) {
+    for (int h = h_first; h < H; h += h_step) {
       const uint16_t* src = src_c + (long long)h * s_head;
       uint16_t* dst = dst_c + (size_t)h * d;
       const uint4 x1 = __ldg(reinterpret_cast<const uint4*>(src));
@@ -75,10 +77,11 @@ __global__ void __launch_bounds__(256, 4) rope_rows_kernel(const uint16_t* __res
 
 void launch_rope_rows(const void* x, const long long x_stride[3], void* y, const double2* tab, const float4* tab_hi,
                       const float4* tab_lo, int C, int L, int H, int d, cudaStream_t st) {
-  const long long n = (long long)L * (d / 16);
-  // enough blocks in flight to cover the memory latency: split the chunks over gridDim.y when L alone is short
-  int ny = C < 64 ? C : 64;
-  dim3 grid((unsigned)((n + 255) / 256), (unsigned)ny);
+  const int bx = (L + 7) / 8;                               // 8 positions per block
+  // a slice of the chunks per block: the table entries are reused over the slice; enough blocks to fill the GPU
+  int ny = (4736 + bx - 1) / bx;
+  ny = ny < 1 ? 1 : (ny > C ? C : ny);
+  dim3 grid((unsigned)bx, (unsigned)ny);
   note_launch();
   rope_rows_kernel<<<grid, 256, 0, st>>>((const uint16_t*)x, x_stride[0], x_stride[1], x_stride[2], (uint16_t*)y, tab_hi,
                                          tab_lo, tab, C, L, H, d);

@@ -58,7 +58,12 @@ def test_workspace_queries_are_host_only(lib):
     assert binding.chunk_prefill_attn_workspace_bytes(1, 64, 64, 4, 2, 64) == 0        # no context token left
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 2, 96) == 0       # head size
     assert binding.chunk_prefill_attn_workspace_bytes(1, 256, 16, 4, 3, 64) == 0       # Hq % Hkv
-    assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 128, 16384) > 0
+    # a batch whose 256-row groups fill the CTA pairs: counter, the three cos/sin tables of the window and the rotated
+    # window queries; no per-split partial results
+    assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 128, 16384) == 256 + 64 * 64 * 16 + 2 * 64 * 32 * 16 + 64 * 64 * 32 * 128 * 2
+    # one sequence: keys split over the CTAs, fp32 partial outputs and (max, sum) per split
+    one = binding.parallel_attn_workspace_bytes(1, 64, 32, 8, 128, 16384)
+    assert one > 256 + 64 * 64 * 16 + 32 * 64 * 128 * 4 * 2 and (one - 256 - 64 * 64 * 16) % (32 * 64 * (128 + 2) * 4) == 0
     assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 100, 16384) == 0
 
 

@@ -25,6 +25,12 @@ def _bits(rng, shape):
     (2, 1, 8, 2, 128, 3000, 8191, 5e5),       # decoding step: one query token over the cache (+ its own key)
     (3, 2, 4, 4, 64, 500, 4094, 1e4),         # two query tokens, MHA
     (1, 4, 32, 8, 128, 16384, 8188, 5e5),     # four query tokens over a 16K cache, Llama-3 heads
+    # batches whose 256-row groups fill the CTA pairs (head size 128, G*w a multiple of 256): the pair kernel
+    (8, 64, 32, 8, 128, 300, 8128, 5e5),      # 64 groups, ragged last cache tile
+    (15, 64, 32, 8, 128, 256, 8128, 5e5),     # 120 groups: two rounds per pair, cache of whole tiles
+    (28, 32, 16, 2, 128, 520, 100, 1e4),      # G = 8, w = 32: four heads per CTA
+    (16, 128, 8, 2, 128, 130, 0, 1e4),        # G*w = 512: two groups per kv-head, one head per CTA, two keys in the last tile
+    (60, 8, 32, 1, 128, 129, 5, 1e4),         # smallest window of that kernel: sixteen heads per CTA
 ])
 def test_parallel_attn_shapes(B, w, Hq, Hkv, d, Nk, q_pos0, theta):
     import paper_2502_14317_b200 as pc
