@@ -541,7 +541,8 @@ def _extra_parallel(pc, torch, dev, peaks, g, out, B=64):
     out["parallel_attn_cfg4" if B == 64 else "parallel_attn_cfg4_B%d" % B] = {"us": us, "tflops": flops / us / 1e6, "kv_gbs": kv_bytes / us / 1e3,
                                  "frac_of_measured_bf16_burst": flops / us / 1e6 / peaks["bf16_tflops"],
                                  "frac_of_measured_hbm": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
-                                 "flops": flops, "kv_bytes": kv_bytes, "l2": "4.3 GB of K/V per call, larger than L2"}
+                                 "flops": flops, "kv_bytes": kv_bytes, "l2": "%.1f GB of K/V per call, larger than L2" % (kv_bytes / 1e9),
+                                 "note": "runs unsplit on CTA pairs when the batch fills them (else key splits + merge)"}
     # ---- decoding step over the same caches: one query token per sequence (w = 1), HBM-bound
     q1 = torch.randn((B, 1, Hq, d), device=dev, generator=g).bfloat16()
     k1 = torch.randn((B, 1, Hkv, d), device=dev, generator=g).bfloat16()
@@ -555,7 +556,7 @@ def _extra_parallel(pc, torch, dev, peaks, g, out, B=64):
     us = _time_us(torch, run_dec, reps=10)
     out["decode_step_cfg4_caches"] = {"us": us, "kv_gbs": kv_bytes / us / 1e3,
                                       "frac_of_measured_hbm": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
-                                      "kv_bytes": kv_bytes, "note": "pc_parallel_attn with w = 1, B = 64, Nk = 16384"}
+                                      "kv_bytes": kv_bytes, "note": "pc_parallel_attn with w = 1, B = %d, Nk = %d" % (B, Nk)}
 
 
 def _extra_select(pc, torch, dev, peaks, g, out, n_chunks):

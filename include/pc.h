@@ -278,7 +278,10 @@ PC_API int32_t pc_queue_emit(const int32_t* q_chunk, int32_t m, int32_t Hkv, int
  * For each of B sequences: the w window queries (rotated here at positions
  * q_pos0..q_pos0+w-1, rounded to bf16) attend to all Nk cache entries of their kv-head
  * (every kept key precedes the window, so no mask) and causally to the window's own w
- * keys.  Keys arrive already rotated.  Split over key ranges with an fp32 merge.
+ * keys.  Keys arrive already rotated.  Small batches are split over key ranges with an fp32
+ * merge; head size 128 with G * w a multiple of 256 and enough (sequence, kv-head) groups to fill the
+ * GPU runs unsplit, one 256-row group per CTA pair (the workspace then also holds the rotated
+ * queries, B * w * Hq * d * 2 bytes).
  * q_win [B,w,Hq,d]; k_cache, v_cache [B,Hkv,Nk,d]; k_win, v_win [B,w,Hkv,d];
  * out [B,w,Hq,d] bf16; lse_out [B,Hq,w] fp32 natural log (may be NULL).  All contiguous.
  * Here w may be any power of two in [1, 128]: w = 1 is a decoding step over the compressed
@@ -306,13 +309,14 @@ PC_API int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, i
  * allocation may cause.  Such callers can still pass inputs and outputs they already
  * hold, but have nowhere to get a workspace from.
  *
- * The scratch (work counter, window cos/sin table, per-split partial results) is a
+ * The scratch (work counter, window cos/sin tables, rotated queries or per-split partial results) is a
  * fixed array of PC_STATIC_SCRATCH_BYTES inside the library image.  Consequences:
  *   - every GPU on which the library is loaded gives up that much memory until the
  *     process exits, whether or not this call is ever used;
  *   - a shape whose pc_parallel_attn_workspace_bytes exceeds the array is refused with
  *     PC_ERR_SCRATCH_LIMIT before anything is launched (B = 1 with tens of thousands of
- *     cached keys splits widely and can exceed it; batches of sequences need little);
+ *     cached keys splits widely and can exceed it; so can a large batch, whose rotated
+ *     window queries live there: B * w * Hq * d * 2 bytes);
  *   - all calls on a device share the one array and it keeps whatever the previous
  *     call left there.  The call clears the part that has to start at zero (the work
  *     counter) on `stream` itself.  Two calls whose kernels can overlap on the GPU

@@ -2,7 +2,7 @@
 // because they are not allowed to allocate device memory at the point of the call
 // (a serving loop that fixed its memory plan at start-up, a plug-in running inside
 // somebody else's allocator, code between a framework's "no allocation" markers).
-// The scratch of the split-K attention (work counter, window cos/sin table, per-split
+// The scratch of the attention (work counter, window cos/sin tables, rotated queries or per-split
 // partial outputs) lives in one array that is part of the library image instead.
 //
 // The array's name is only a handle on the host: its device address is asked for once
