@@ -278,10 +278,10 @@ PC_API int32_t pc_queue_emit(const int32_t* q_chunk, int32_t m, int32_t Hkv, int
  * For each of B sequences: the w window queries (rotated here at positions
  * q_pos0..q_pos0+w-1, rounded to bf16) attend to all Nk cache entries of their kv-head
  * (every kept key precedes the window, so no mask) and causally to the window's own w
- * keys.  Keys arrive already rotated.  Small batches are split over key ranges with an fp32
+ * keys.  Keys arrive already rotated; the queries are rotated into the workspace first
+ * (B * w * Hq * d * 2 bytes of it).  Small batches are split over key ranges with an fp32
  * merge; head size 128 with G * w a multiple of 256 and enough (sequence, kv-head) groups to fill the
- * GPU runs unsplit, one 256-row group per CTA pair (the workspace then also holds the rotated
- * queries, B * w * Hq * d * 2 bytes).
+ * GPU runs unsplit, one 256-row group per CTA pair.
  * q_win [B,w,Hq,d]; k_cache, v_cache [B,Hkv,Nk,d]; k_win, v_win [B,w,Hkv,d];
  * out [B,w,Hq,d] bf16; lse_out [B,Hq,w] fp32 natural log (may be NULL).  All contiguous.
  * Here w may be any power of two in [1, 128]: w = 1 is a decoding step over the compressed

@@ -375,11 +375,13 @@ struct ParallelPlan {
   size_t off_counter, off_table, off_table_hi, off_table_lo, off_qrot, off_ml, off_o, total;
 };
 
-// Split the keys so that the persistent grid has a few items per SM; every split keeps at
-// least two cache tiles.  The plan depends only on the sizes and the SM count.
+// The plan depends only on the sizes and the SM count.
 // Head size 128 with whole 256-row groups per (sequence, kv-head) runs on CTA pairs, one group per pair and
 // item, without a key split, when the groups fill the pairs' rounds to three quarters or more (the pair kernel is
 // about a third faster per tile, a partly filled last round costs it that advantage).
+// Otherwise the single-CTA kernel splits the keys.  The number of splits minimises a cost model in units of one
+// key tile: rounds of the persistent grid x (fixed cost of an item - query load, pipeline fill, write-out of
+// the partial result - of about four tiles + tiles per split).
 ParallelPlan parallel_plan(int B, int w, int Hq, int Hkv, int d, int Nk, int sm_count) {
   ParallelPlan p;
   const int G = Hq / Hkv;
@@ -398,24 +400,28 @@ ParallelPlan parallel_plan(int B, int w, int Hq, int Hkv, int d, int Nk, int sm_
       p.n_rg_pair = G * w / 256;
     }
   }
-  long long want = (4LL * sm_count + base - 1) / base;
-  long long cap = p.n_cache_tiles / 2;
-  if (cap < 1) cap = 1;
-  if (want > cap) want = cap;
-  if (want < 1) want = 1;
-  if (p.pair) want = 1;
-  p.tiles_per_split = (int)((p.n_cache_tiles + want - 1) / want);
+  p.tiles_per_split = p.n_cache_tiles;
+  if (!p.pair) {
+    constexpr long long ITEM_COST_TILES = 4;
+    long long best = -1;
+    int max_split = p.n_cache_tiles / 2;                       // every split keeps at least two cache tiles
+    max_split = max_split < 1 ? 1 : (max_split > 64 ? 64 : max_split);
+    for (int s = 1; s <= max_split; ++s) {
+      const int tps = (p.n_cache_tiles + s - 1) / s;
+      const int ns = (p.n_cache_tiles + tps - 1) / tps;
+      const long long rounds = (base * ns + sm_count - 1) / sm_count;
+      const long long cost = rounds * (ITEM_COST_TILES + tps + (ns > 1 ? 1 : 0));   // a split run also pays for the merge
+      if (best < 0 || cost < best) { best = cost; p.tiles_per_split = tps; }
+    }
+  }
   if (p.tiles_per_split < 1) p.tiles_per_split = 1;
   p.n_split = p.n_cache_tiles > 0 ? (p.n_cache_tiles + p.tiles_per_split - 1) / p.tiles_per_split : 1;
   size_t off = 0;
   p.off_counter = off; off += ALIGN;
   p.off_table = off; off += align_up((size_t)w * (d / 2) * sizeof(double2));
-  p.off_table_hi = off;
-  if (p.pair) off += align_up((size_t)w * (d / 4) * sizeof(float4));
-  p.off_table_lo = off;
-  if (p.pair) off += align_up((size_t)w * (d / 4) * sizeof(float4));
-  p.off_qrot = off;
-  if (p.pair) off += align_up((size_t)B * w * Hq * d * 2);
+  p.off_table_hi = off; off += align_up((size_t)w * (d / 4) * sizeof(float4));
+  p.off_table_lo = off; off += align_up((size_t)w * (d / 4) * sizeof(float4));
+  p.off_qrot = off; off += align_up((size_t)B * w * Hq * d * 2);
   p.off_ml = off;
   if (p.n_split > 1) off += align_up((size_t)B * Hq * p.n_split * w * 2 * sizeof(float));
   p.off_o = off;
@@ -478,14 +484,15 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   const uint32_t box_kc[4] = {64, 128, 1, 1};
   const uint32_t box_kw[4] = {64, 1, 128, 1};
 
+  // rotated queries first (the same pass that serves the chunk-local kernels)
+  float4* table_hi = reinterpret_cast<float4*>(ws + plan.off_table_hi);
+  float4* table_lo = reinterpret_cast<float4*>(ws + plan.off_table_lo);
+  void* q_rot = ws + plan.off_qrot;
+  pc::launch_rope_table(table, table_hi, table_lo, w, d, (double)rope_theta, q_pos0, st);
+  const long long q_stride[3] = {(long long)w * Hq * d, (long long)Hq * d, (long long)d};
+  pc::launch_rope_rows(q_win, q_stride, q_rot, table, table_hi, table_lo, B, w, Hq, d, st);
+
   if (plan.pair) {
-    // rotated queries first (the same pass that serves the chunk-local kernel), then the pair kernel
-    float4* table_hi = reinterpret_cast<float4*>(ws + plan.off_table_hi);
-    float4* table_lo = reinterpret_cast<float4*>(ws + plan.off_table_lo);
-    void* q_rot = ws + plan.off_qrot;
-    pc::launch_rope_table(table, table_hi, table_lo, w, d, (double)rope_theta, q_pos0, st);
-    const long long q_stride[3] = {(long long)w * Hq * d, (long long)Hq * d, (long long)d};
-    pc::launch_rope_rows(q_win, q_stride, q_rot, table, table_hi, table_lo, B, w, Hq, d, st);
     CUtensorMap pm[6];
     const uint32_t box_kch[4] = {64, 64, 1, 1};
     const uint32_t box_kwh[4] = {64, 1, 64, 1};
@@ -509,7 +516,7 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   }
 
   CUtensorMap maps[5];
-  if (!pc::make_tmap_bf16_4d(&maps[0], q_win, qw_dims, qw_str, box_qw) ||
+  if (!pc::make_tmap_bf16_4d(&maps[0], q_rot, qw_dims, qw_str, box_qw) ||
       !pc::make_tmap_bf16_4d(&maps[1], k_cache, kc_dims, kc_str, box_kc) ||
       !pc::make_tmap_bf16_4d(&maps[2], v_cache, kc_dims, kc_str, box_kc) ||
       !pc::make_tmap_bf16_4d(&maps[3], k_win, kw_dims, kw_str, box_kw) ||
@@ -517,7 +524,6 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
     return PC_ERR_CUDA;
 
   if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return PC_ERR_CUDA;
-  pc::launch_rope_table(table, nullptr, nullptr, w, d, (double)rope_theta, q_pos0, st);
 
   pc::ParallelParams prm;
   prm.B = B; prm.w = w; prm.Hq = Hq; prm.Hkv = Hkv; prm.Nk = Nk;
@@ -525,7 +531,6 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   prm.n_cache_tiles = plan.n_cache_tiles; prm.n_split = plan.n_split; prm.tiles_per_split = plan.tiles_per_split;
   const double scale = softmax_scale > 0.0f ? (double)softmax_scale : 1.0 / std::sqrt((double)d);
   prm.scale_log2 = (float)(scale * 1.4426950408889634);
-  prm.rope_tab = table;
   prm.part_ml = reinterpret_cast<float*>(ws + plan.off_ml);
   prm.part_o = reinterpret_cast<float*>(ws + plan.off_o);
   prm.out = static_cast<__nv_bfloat16*>(out);

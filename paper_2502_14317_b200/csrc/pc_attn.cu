@@ -41,10 +41,10 @@ constexpr float LAZY_RESCALE = 8.0f;        // log2 units
 constexpr int ITEM_DONE = -1;
 
 // where-codes stored in the status word when a wait gives up
-enum { W_ITEM = 101, W_QFULL, W_QROT, W_QFREE, W_KVFULL, W_KVFREE, W_SFULL, W_PFULL, W_OFULL, W_ACCFREE, W_TFULL, W_TFREE, W_TURN, W_PHALF };
+enum { W_ITEM = 101, W_QFULL, W_QROT /* unused, keeps the later codes */, W_QFREE, W_KVFULL, W_KVFREE, W_SFULL, W_PFULL, W_OFULL, W_ACCFREE, W_TFULL, W_TFREE, W_TURN, W_PHALF };
 
 struct __align__(16) Misc {
-  uint64_t q_full[2], q_rot[2], q_free[2];
+  uint64_t q_full[2], q_free[2];
   uint64_t kv_full[NS], kv_free[NS];
   uint64_t s_full[2], p_half[2], p_full[2], o_full[2], acc_free[2];
   uint64_t item_full[2], item_empty[2];
@@ -162,37 +162,6 @@ __device__ __forceinline__ SubItem decode_sub(const Sched& s, int hkv, int withi
   return it;
 }
 
-// ------------------------------------------------------------------ RoPE of a query row in shared memory
-// Row `row` of a 128-byte-swizzled [128 x D] bf16 tile; pairs (t, t + D/2); fp64 math, one rounding.
-template <int D>
-__device__ __forceinline__ void rope_row_smem(uint8_t* tile, int row, const double2* __restrict__ tab_row) {
-#pragma unroll 1
-  for (int cidx = 0; cidx < D / 16; ++cidx) {
-    uint8_t* lo_p = tile + sw128_offset(row, cidx);
-    uint8_t* hi_p = (D == 128) ? tile + 16384 + sw128_offset(row, cidx) : tile + sw128_offset(row, cidx + 4);
-    const uint4 lo = *reinterpret_cast<const uint4*>(lo_p);
-    const uint4 hi = *reinterpret_cast<const uint4*>(hi_p);
-    const uint32_t lo_w[4] = {lo.x, lo.y, lo.z, lo.w}, hi_w[4] = {hi.x, hi.y, hi.z, hi.w};
-    uint32_t out_lo[4], out_hi[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint32_t rl = 0, rh = 0;
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const double x1 = (double)__uint_as_float(((lo_w[i] >> (16 * e)) & 0xFFFFu) << 16);
-        const double x2 = (double)__uint_as_float(((hi_w[i] >> (16 * e)) & 0xFFFFu) << 16);
-        const double2 t = tab_row[cidx * 8 + 2 * i + e];
-        rl |= (uint32_t)f64_to_bf16_rne(x1 * t.x - x2 * t.y) << (16 * e);
-        rh |= (uint32_t)f64_to_bf16_rne(x2 * t.x + x1 * t.y) << (16 * e);
-      }
-      out_lo[i] = rl;
-      out_hi[i] = rh;
-    }
-    *reinterpret_cast<uint4*>(lo_p) = make_uint4(out_lo[0], out_lo[1], out_lo[2], out_lo[3]);
-    *reinterpret_cast<uint4*>(hi_p) = make_uint4(out_hi[0], out_hi[1], out_hi[2], out_hi[3]);
-  }
-}
-
 // One arrival for a whole warp (an arrival per thread costs the barrier 32 serialised shared-memory operations).
 __device__ __forceinline__ void warp_arrive(uint64_t* bar) {
   __syncwarp();
@@ -307,7 +276,7 @@ __device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint3
 
 // ------------------------------------------------------------------ per-role state
 struct Waits {                                 // how many times each barrier has been used by this role
-  uint32_t q[2] = {0, 0};                      // q_full / q_rot / q_free (one use per block load)
+  uint32_t q[2] = {0, 0};                      // q_full / q_free (one use per block load)
   uint32_t kv = 0;                             // ring position (monotone)
   uint32_t s[2] = {0, 0}, p[2] = {0, 0}, o[2] = {0, 0}, acc[2] = {0, 0};   // p counts p_half and p_full alike
   uint32_t t[2] = {0, 0};
@@ -330,7 +299,7 @@ struct Ctx {
 __device__ __forceinline__ void init_barriers(Misc& mi, int wait_kcycles) {
 #pragma unroll
   for (int b = 0; b < 2; ++b) {
-    mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_rot[b], 4); mbar_init(&mi.q_free[b], 1);        // groups arrive once per warp
+    mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_free[b], 1);
     mbar_init(&mi.s_full[b], 1); mbar_init(&mi.p_half[b], 4); mbar_init(&mi.p_full[b], 4); mbar_init(&mi.o_full[b], 1);
     mbar_init(&mi.acc_free[b], 4);
     mbar_init(&mi.item_full[b], 1); mbar_init(&mi.item_empty[b], 10);      // 8 softmax warps + 2 issuer threads
@@ -410,7 +379,7 @@ __device__ __forceinline__ void turn_pass(const Ctx& cx, Waits& wt, int b) {
 // walks the ring, takes its turns and releases the stages it does not use, so that both
 // issuers arrive once on every kv_free barrier and the token keeps alternating.
 template <int D>
-__device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b, bool has_b, int nb_b, int n, bool q_rotated_here) {
+__device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b, bool has_b, int nb_b, int n) {
   using C = Cfg<D>;
   Misc& mi = *cx.mi;
   const uint32_t ring_u32 = smem_u32(cx.ring);
@@ -421,9 +390,8 @@ __device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b,
     mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
 #pragma unroll
     for (int e = 0; e < 2; ++e) mbar_wait(&mi.t_free[e], free_par(wt.t[e]), cx.abort_flag, cx.status, W_TFREE);
-    // the query block is ready: rotated in shared memory by the softmax group (parallel attention), or, already
-    // rotated in global memory, as soon as its copy has landed (chunk prefill)
-    mbar_wait(q_rotated_here ? &mi.q_rot[b] : &mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QROT);
+    // the query block (rotated by the pre-pass, in global memory) is ready as soon as its copy has landed
+    mbar_wait(&mi.q_full[b], full_par(wt.q[b]), cx.abort_flag, cx.status, W_QFULL);
     ++wt.q[b];
   }
   {  // S(0)
@@ -614,7 +582,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const bool has_b = (b == 0) || it.hB >= 0;
           const int nb_b = (b == 0) ? it.tA + 1 : (it.hB >= 0 ? it.tB + 1 : 0);
           const int n = (it.hB >= 0 ? it.tB : it.tA) + 1;
-          mma_flash_block<D>(cx, wt, b, has_b, nb_b, n, false);
+          mma_flash_block<D>(cx, wt, b, has_b, nb_b, n);
         }
         if (within == 0) {
           // ---- score sweep: this issuer computes the columns of its own block (window rows b*128..)
@@ -778,7 +746,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 // ====================================================================================
 //                          PARALLEL (GLOBAL) ATTENTION KERNEL
 // ====================================================================================
-// Item = (sequence, kv-head, row group, key split).  The rows of an item are the w window
+// Queries arrive rotated (RoPE pre-pass).  Item = (sequence, kv-head, row group, key split).  The rows of an item are the w window
 // queries of up to 256/w q-heads of one kv-head, packed head-major into the two 128-row
 // blocks; both blocks stream the same cache tiles, and the last split appends the
 // window's own keys (causal inside the window).
@@ -873,7 +841,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
         if (item == ITEM_DONE) break;
         const Dec d = decode(item);
         const bool has_b = d.rows[b] > 0;
-        mma_flash_block<D>(cx, wt, b, has_b, has_b ? d.n : 0, d.n, true);
+        mma_flash_block<D>(cx, wt, b, has_b, has_b ? d.n : 0, d.n);
       }
       mma_commit(&mi.mma_done);
     }
@@ -883,8 +851,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
     const int r = tid & 127;
     const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tS = cx.tmem + b * 128 + lane_sel, tO = cx.tmem + 256 + b * 128 + lane_sel;
-    uint8_t* const myQ = b ? cx.sQ[1] : cx.sQ[0];
-    uint32_t n_q = 0, n_s = 0, n_o = 0;
+    uint32_t n_s = 0, n_o = 0;
     const int wi = r % prm.w;                                 // window index of this row (128 % w == 0)
     while (true) {
       const int item = consumer_next_item(cx, wt, true);
@@ -892,11 +859,6 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
       const Dec d = decode(item);
       const int rows_b = b ? d.rows[1] : d.rows[0];
       if (rows_b == 0) continue;
-      mbar_wait(&mi.q_full[b], full_par(n_q), cx.abort_flag, cx.status, W_QFULL);
-      ++n_q;
-      if (r < rows_b) rope_row_smem<D>(myQ, r, prm.rope_tab + (size_t)wi * (D / 2));
-      fence_proxy_async_smem();
-      warp_arrive(&mi.q_rot[b]);
       float m_used, l_run;
       wg_flash_loop<D>(cx, n_s, n_o, b, tS, tO, d.n, prm.scale_log2,
                        [&](int jj) {

@@ -31,7 +31,6 @@ struct ParallelParams {
   int Gs, n_rg;                  // q-heads per row group (Gs * w <= 256), row groups per kv-head
   int n_cache_tiles, n_split, tiles_per_split;
   float scale_log2;
-  const double2* rope_tab;       // [w][d/2] for positions q_pos0 .. q_pos0 + w - 1
   float* part_o;                 // [B,Hq,n_split,w,d] fp32 unnormalised partial outputs (n_split > 1)
   float* part_ml;                // [B,Hq,n_split,w,2] (running max in log2 units, sum)
   __nv_bfloat16* out;            // [B,w,Hq,d]
@@ -41,7 +40,7 @@ struct ParallelParams {
   int wait_kcycles;              // limit of every device-side wait, in units of 1024 cycles
 };
 
-// maps: q_win (w-row box), k_cache, v_cache (128-key box), k_win, v_win (128-row box over w tokens)
+// maps: rotated q_win (w-row box), k_cache, v_cache (128-key box), k_win, v_win (128-row box over w tokens)
 cudaError_t launch_parallel_attn(const CUtensorMap* maps, const ParallelParams& prm, int d, int grid, cudaStream_t st);
 
 // Parallel attention on CTA pairs (head size 128, G * w a multiple of 256, no key split): every pair takes the

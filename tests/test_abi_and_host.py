@@ -61,9 +61,10 @@ def test_workspace_queries_are_host_only(lib):
     # a batch whose 256-row groups fill the CTA pairs: counter, the three cos/sin tables of the window and the rotated
     # window queries; no per-split partial results
     assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 128, 16384) == 256 + 64 * 64 * 16 + 2 * 64 * 32 * 16 + 64 * 64 * 32 * 128 * 2
-    # one sequence: keys split over the CTAs, fp32 partial outputs and (max, sum) per split
-    one = binding.parallel_attn_workspace_bytes(1, 64, 32, 8, 128, 16384)
-    assert one > 256 + 64 * 64 * 16 + 32 * 64 * 128 * 4 * 2 and (one - 256 - 64 * 64 * 16) % (32 * 64 * (128 + 2) * 4) == 0
+    # one sequence: keys split over the CTAs (16 splits of 8 tiles: one item per SM), fp32 partial outputs and
+    # (max, sum) per split besides the tables and the rotated queries
+    fixed = 256 + 64 * 64 * 16 + 2 * 64 * 32 * 16 + 1 * 64 * 32 * 128 * 2
+    assert binding.parallel_attn_workspace_bytes(1, 64, 32, 8, 128, 16384) == fixed + 16 * 32 * 64 * (128 + 2) * 4
     assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 100, 16384) == 0
 
 
