@@ -41,6 +41,10 @@ void launch_rope_table(double2* tab, float4* tab_hi, float4* tab_lo, int n_pos, 
 // piece of the token's row (1 KB for d = 128), and a block of 8 warps streams 8 adjacent rows: the DRAM pages
 // are walked front to back, as a copy would.  The table entries of (position, pairs) stay in registers across
 // the heads and across the chunks of the block's slice.
+// Outputs that the fp32 arithmetic cannot decide (about one in 1300) are redone exactly by the whole warp: the
+// sixteen outputs of an undecided lane go to sixteen lanes, one each, and are patched into the row after the
+// vector store.  (Handling them in the lane that found them would make a third of the warp's passes wait for one
+// lane's slow path.)
 __global__ void __launch_bounds__(256, 4) rope_rows_kernel(const uint16_t* __restrict__ x, long long s_chunk, long long s_tok,
                                                            long long s_head, uint16_t* __restrict__ y,
                                                            const float4* __restrict__ tab_hi, const float4* __restrict__ tab_lo,
@@ -49,28 +53,71 @@ __global__ void __launch_bounds__(256, 4) rope_rows_kernel(const uint16_t* __res
   const int groups = half / 8;                              // 16-byte groups per half row (4 or 8)
   const int lane = threadIdx.x & 31;
   const int p = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (p >= L) return;
+  if (p >= L) return;                                       // whole warps leave together
   const int g = lane % groups, h_first = lane / groups, h_step = 32 / groups;
-  const size_t e0 = (size_t)p * half + g * 8;               // first pair of this thread in the tables
+  const size_t row0 = (size_t)p * half;                     // first pair of this position in the tables
+  const float4* hi_row = tab_hi + row0 / 2;
+  const float4* lo_row = tab_lo + row0 / 2;
+  const double2* d_row = tab + row0;
   float4 hi[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) hi[i] = __ldg(tab_hi + e0 / 2 + i);
+  for (int i = 0; i < 4; ++i) hi[i] = __ldg(hi_row + g * 4 + i);
+  const long long step_src = (long long)h_step * s_head;
+  const int n_pass = (H + h_step - 1) / h_step;
   for (int c = blockIdx.y; c < C; c += gridDim.y) {
-    const uint16_t* src_c = x + (long long)c * s_chunk + (long long)p * s_tok + g * 8;
-    uint16_t* dst_c = y + ((size_t)c * L + p) * H * d + g * 8;
+    const uint16_t* src = x + (long long)c * s_chunk + (long long)p * s_tok + (long long)h_first * s_head + g * 8;
+    uint16_t* const dst_tok = y + ((size_t)c * L + p) * H * d;
+    uint16_t* dst = dst_tok + (size_t)h_first * d + g * 8;
+    uint4 n1 = make_uint4(0, 0, 0, 0), n2 = make_uint4(0, 0, 0, 0);
+    if (h_first < H) {
+      n1 = __ldg(reinterpret_cast<const uint4*>(src));
+      n2 = __ldg(reinterpret_cast<const uint4*>(src + half));
+    }
 #pragma unroll 1
-    for (int h = h_first; h < H; h += h_step) {
-      const uint16_t* src = src_c + (long long)h * s_head;
-      uint16_t* dst = dst_c + (size_t)h * d;
-      const uint4 x1 = __ldg(reinterpret_cast<const uint4*>(src));
-      const uint4 x2 = __ldg(reinterpret_cast<const uint4*>(src + half));
+    for (int ps = 0; ps < n_pass; ++ps, src += step_src, dst += (size_t)h_step * d) {
+      const bool active = h_first + ps * h_step < H;
+      const uint4 x1 = n1, x2 = n2;
+      if (h_first + (ps + 1) * h_step < H) {                // the next pass's row is in flight during this one's arithmetic
+        n1 = __ldg(reinterpret_cast<const uint4*>(src + step_src));
+        n2 = __ldg(reinterpret_cast<const uint4*>(src + step_src + half));
+      } else {
+        n1 = make_uint4(0, 0, 0, 0); n2 = make_uint4(0, 0, 0, 0);
+      }
       uint4 y1, y2;
-      rope_two_pairs(x1.x, x2.x, hi[0], tab_lo + e0 / 2 + 0, tab + e0 + 0, y1.x, y2.x);
-      rope_two_pairs(x1.y, x2.y, hi[1], tab_lo + e0 / 2 + 1, tab + e0 + 2, y1.y, y2.y);
-      rope_two_pairs(x1.z, x2.z, hi[2], tab_lo + e0 / 2 + 2, tab + e0 + 4, y1.z, y2.z);
-      rope_two_pairs(x1.w, x2.w, hi[3], tab_lo + e0 / 2 + 3, tab + e0 + 6, y1.w, y2.w);
-      *reinterpret_cast<uint4*>(dst) = y1;
-      *reinterpret_cast<uint4*>(dst + half) = y2;
+      uint32_t amb = rope_two_pairs_fast(x1.x, x2.x, hi[0], y1.x, y2.x);
+      amb |= rope_two_pairs_fast(x1.y, x2.y, hi[1], y1.y, y2.y);
+      amb |= rope_two_pairs_fast(x1.z, x2.z, hi[2], y1.z, y2.z);
+      amb |= rope_two_pairs_fast(x1.w, x2.w, hi[3], y1.w, y2.w);
+      if (active) {
+        *reinterpret_cast<uint4*>(dst) = y1;
+        *reinterpret_cast<uint4*>(dst + half) = y2;
+      }
+      unsigned todo = __ballot_sync(0xFFFFFFFFu, active && amb != 0u);
+      if (todo != 0u) {                                     // warp-uniform
+        __syncwarp();                                       // the vector stores above precede the patches below
+        const int t = (lane >> 1) & 7, second = lane & 1;   // lanes 0..15: pair t of the undecided lane, first / second output
+        do {
+          const int srcl = __ffs(todo) - 1;
+          todo &= todo - 1;
+          const uint32_t w1[4] = {__shfl_sync(0xFFFFFFFFu, x1.x, srcl), __shfl_sync(0xFFFFFFFFu, x1.y, srcl),
+                                  __shfl_sync(0xFFFFFFFFu, x1.z, srcl), __shfl_sync(0xFFFFFFFFu, x1.w, srcl)};
+          const uint32_t w2[4] = {__shfl_sync(0xFFFFFFFFu, x2.x, srcl), __shfl_sync(0xFFFFFFFFu, x2.y, srcl),
+                                  __shfl_sync(0xFFFFFFFFu, x2.z, srcl), __shfl_sync(0xFFFFFFFFu, x2.w, srcl)};
+          if (lane < 16) {
+            const int wsel = t >> 1;
+            const uint32_t u1 = wsel == 0 ? w1[0] : wsel == 1 ? w1[1] : wsel == 2 ? w1[2] : w1[3];
+            const uint32_t u2 = wsel == 0 ? w2[0] : wsel == 1 ? w2[1] : wsel == 2 ? w2[2] : w2[3];
+            const float a = __uint_as_float((t & 1) ? (u1 & 0xFFFF0000u) : (u1 << 16));
+            const float b = __uint_as_float((t & 1) ? (u2 & 0xFFFF0000u) : (u2 << 16));
+            const int sg = srcl % groups, sh = srcl / groups + ps * h_step;      // pair group and head of that lane
+            const int pair = sg * 8 + t;
+            const uint32_t r = second ? rope_one_exact(b, -a, pair, hi_row, lo_row, d_row)
+                                      : rope_one_exact(a, b, pair, hi_row, lo_row, d_row);
+            dst_tok[(size_t)sh * d + (second ? half : 0) + pair] = (uint16_t)r;
+          }
+        } while (todo != 0u);
+        __syncwarp();
+      }
     }
   }
 }

@@ -47,30 +47,27 @@ __device__ __forceinline__ uint32_t rope_out_dd(float a, float b, float ch, floa
 // Table layout of the fp32 heads and tails: one float4 per TWO consecutive pairs (2i, 2i + 1) of a position,
 // (cos_2i, cos_2i+1, sin_2i, sin_2i+1), so that the packed fp32 instructions find their operands in register pairs.
 //
-// Levels 2 and 3 for the two pairs (a0, b0), (a1, b1) at the table entry `hi` (heads), `lo_p` (tails), `d_p` (fp64,
-// (cos, sin) per pair).  Returns the bf16 bits: y1 = a c - b s of both pairs in lo_out, y2 = b c + a s in up_out.
-__device__ __noinline__ static void rope_pairs_exact(float a0, float a1, float b0, float b1, float4 hi,
-                                                     const float4* __restrict__ lo_p, const double2* __restrict__ d_p,
-                                                     uint32_t& lo_out, uint32_t& up_out) {
-  const float4 lo = __ldg(lo_p);
-  uint32_t y1a = rope_out_dd(a0, b0, hi.x, hi.z, lo.x, lo.z), y2a = rope_out_dd(b0, -a0, hi.x, hi.z, lo.x, lo.z);
-  uint32_t y1b = rope_out_dd(a1, b1, hi.y, hi.w, lo.y, lo.w), y2b = rope_out_dd(b1, -a1, hi.y, hi.w, lo.y, lo.w);
-  if ((y1a | y2a | y1b | y2b) == 0xFFFFFFFFu) {
-    const double2 t0 = __ldg(d_p), t1 = __ldg(d_p + 1);
-    const double da0 = (double)a0, da1 = (double)a1, db0 = (double)b0, db1 = (double)b1;
-    if (y1a == 0xFFFFFFFFu) y1a = f64_to_bf16_rne(da0 * t0.x - db0 * t0.y);
-    if (y2a == 0xFFFFFFFFu) y2a = f64_to_bf16_rne(db0 * t0.x + da0 * t0.y);
-    if (y1b == 0xFFFFFFFFu) y1b = f64_to_bf16_rne(da1 * t1.x - db1 * t1.y);
-    if (y2b == 0xFFFFFFFFu) y2b = f64_to_bf16_rne(db1 * t1.x + da1 * t1.y);
+// Levels 2 and 3 for ONE output y = a * c - b * s (pass (b, -a) for the second output of a pair, b c + a s) at
+// table entry `pair` of a position's row: heads in hi_row, tails in lo_row (float4 per two pairs), fp64 (cos, sin)
+// in d_row.  Returns the bf16 bits.
+__device__ __forceinline__ uint32_t rope_one_exact(float a, float b, int pair, const float4* __restrict__ hi_row,
+                                                   const float4* __restrict__ lo_row, const double2* __restrict__ d_row) {
+  const float* h = reinterpret_cast<const float*>(hi_row + (pair >> 1));
+  const float* l = reinterpret_cast<const float*>(lo_row + (pair >> 1));
+  const int e = pair & 1;
+  uint32_t r = rope_out_dd(a, b, __ldg(h + e), __ldg(h + 2 + e), __ldg(l + e), __ldg(l + 2 + e));
+  if (r == 0xFFFFFFFFu) {
+    const double2 t = __ldg(d_row + pair);
+    r = f64_to_bf16_rne((double)a * t.x - (double)b * t.y);
   }
-  lo_out = y1a | (y1b << 16);
-  up_out = y2a | (y2b << 16);
+  return r;
 }
 
-// Two pairs through level 1 (packed fp32 arithmetic); falls back to rope_pairs_exact.  x1w / x2w: the two bf16 of
-// x1 (first half of the row) and of x2 (second half) as they sit in memory; same layout on return.
-__device__ __forceinline__ void rope_two_pairs(uint32_t x1w, uint32_t x2w, float4 hi, const float4* __restrict__ lo_p,
-                                               const double2* __restrict__ d_p, uint32_t& lo_out, uint32_t& up_out) {
+// Two pairs through level 1 (packed fp32 arithmetic).  x1w / x2w: the two bf16 of x1 (first half of the row) and of
+// x2 (second half) as they sit in memory; same layout on return.  Returns non-zero when one of the four outputs is
+// too close to a rounding boundary for level 1 to decide (that output is then not valid yet).
+__device__ __forceinline__ uint32_t rope_two_pairs_fast(uint32_t x1w, uint32_t x2w, float4 hi, uint32_t& lo_out,
+                                                        uint32_t& up_out) {
   const float a0 = __uint_as_float(x1w << 16), a1 = __uint_as_float(x1w & 0xFFFF0000u);
   const float b0 = __uint_as_float(x2w << 16), b1 = __uint_as_float(x2w & 0xFFFF0000u);
   const uint64_t A = pack_f32x2(a0, a1), B = pack_f32x2(b0, b1), NB = pack_f32x2(-b0, -b1);
@@ -82,16 +79,14 @@ __device__ __forceinline__ void rope_two_pairs(uint32_t x1w, uint32_t x2w, float
   const uint64_t NT = pack_f32x2(-2.3841858e-7f * m0, -2.3841858e-7f * m1);
   float p, q;
   unpack_f32x2(add_f32x2(Y1, NT), p, q);
-  const uint32_t lo_dn = pack_bf16x2(p, q);
+  lo_out = pack_bf16x2(p, q);
   unpack_f32x2(add_f32x2(Y1, T), p, q);
   const uint32_t lo_up = pack_bf16x2(p, q);
   unpack_f32x2(add_f32x2(Y2, NT), p, q);
-  const uint32_t up_dn = pack_bf16x2(p, q);
+  up_out = pack_bf16x2(p, q);
   unpack_f32x2(add_f32x2(Y2, T), p, q);
   const uint32_t up_up = pack_bf16x2(p, q);
-  lo_out = lo_dn;
-  up_out = up_dn;
-  if (((lo_dn ^ lo_up) | (up_dn ^ up_up)) != 0u) rope_pairs_exact(a0, a1, b0, b1, hi, lo_p, d_p, lo_out, up_out);
+  return (lo_out ^ lo_up) | (up_out ^ up_up);
 }
 
 }  // namespace pc
