@@ -370,6 +370,8 @@ namespace {
 
 struct ParallelPlan {
   int Gs, n_rg, n_cache_tiles, n_split, tiles_per_split;
+  bool alt;                        // single-CTA kernel, rows of an item fit one block: two streams on alternate key tiles
+  int n_part;                      // partial results to merge per (sequence, q-head)
   bool pair;                       // CTA-pair kernel: 256-row groups, no key split
   int hpc, n_rg_pair;              // pair kernel: q-heads per CTA, 256-row groups per kv-head
   size_t off_counter, off_table, off_table_hi, off_table_lo, off_qrot, off_ml, off_o, total;
@@ -422,10 +424,12 @@ ParallelPlan parallel_plan(int B, int w, int Hq, int Hkv, int d, int Nk, int sm_
   p.off_table_hi = off; off += align_up((size_t)w * (d / 4) * sizeof(float4));
   p.off_table_lo = off; off += align_up((size_t)w * (d / 4) * sizeof(float4));
   p.off_qrot = off; off += align_up((size_t)B * w * Hq * d * 2);
+  p.alt = !p.pair && p.Gs * w <= 128;
+  p.n_part = p.alt ? 2 * p.n_split : p.n_split;
   p.off_ml = off;
-  if (p.n_split > 1) off += align_up((size_t)B * Hq * p.n_split * w * 2 * sizeof(float));
+  if (p.n_part > 1) off += align_up((size_t)B * Hq * p.n_part * w * 2 * sizeof(float));
   p.off_o = off;
-  if (p.n_split > 1) off += align_up((size_t)B * Hq * p.n_split * w * d * sizeof(float));
+  if (p.n_part > 1) off += align_up((size_t)B * Hq * p.n_part * w * d * sizeof(float));
   p.total = off;
   return p;
 }
@@ -529,6 +533,7 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   prm.B = B; prm.w = w; prm.Hq = Hq; prm.Hkv = Hkv; prm.Nk = Nk;
   prm.Gs = plan.Gs; prm.n_rg = plan.n_rg;
   prm.n_cache_tiles = plan.n_cache_tiles; prm.n_split = plan.n_split; prm.tiles_per_split = plan.tiles_per_split;
+  prm.alt = plan.alt ? 1 : 0; prm.n_part = plan.n_part;
   const double scale = softmax_scale > 0.0f ? (double)softmax_scale : 1.0 / std::sqrt((double)d);
   prm.scale_log2 = (float)(scale * 1.4426950408889634);
   prm.part_ml = reinterpret_cast<float*>(ws + plan.off_ml);

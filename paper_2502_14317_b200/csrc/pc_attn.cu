@@ -375,16 +375,20 @@ __device__ __forceinline__ void turn_pass(const Ctx& cx, Waits& wt, int b) {
 }
 
 // issuer of block b: the flash loop over the n K/V tiles of the ring (order K0, V0, K1, V1, ...).
-// Block b takes part in its first nb_b tiles; the issuer of an absent or shorter block still
-// walks the ring, takes its turns and releases the stages it does not use, so that both
-// issuers arrive once on every kv_free barrier and the token keeps alternating.
+// Block b takes part in its first nb_b tiles - or, with `alternate` (the two blocks hold the SAME query rows and
+// share the key tiles of the item between them), in the tiles of parity b.  The issuer of an absent or shorter block
+// still walks the ring, takes its turns and releases the stages it does not use, so that both issuers arrive once
+// on every kv_free barrier and the token keeps alternating.
 template <int D>
-__device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b, bool has_b, int nb_b, int n) {
+__device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b, bool has_b, int nb_b, int n,
+                                                bool alternate = false) {
   using C = Cfg<D>;
   Misc& mi = *cx.mi;
   const uint32_t ring_u32 = smem_u32(cx.ring);
   const uint32_t q_u32 = smem_u32(cx.sQ[b]);
   const uint32_t tS = cx.tmem + b * 128, tO = cx.tmem + 256 + b * 128;
+  auto takes_part = [&](int j) { return has_b && j < n && (alternate ? ((j & 1) == b) : (j < nb_b)); };
+  const int last = alternate ? (((n - 1) & 1) == b ? n - 1 : n - 2) : nb_b - 1;     // last tile of this block
   if (has_b) {
     // accumulator and score buffers of earlier work must have been read out
     mbar_wait(&mi.acc_free[b], free_par(wt.acc[b]), cx.abort_flag, cx.status, W_ACCFREE);
@@ -399,7 +403,7 @@ __device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b,
     mbar_wait(&mi.kv_full[st], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
     ++wt.kv;
     turn_take(cx, wt, b);
-    if (has_b) {
+    if (takes_part(0)) {
       tc_fence_after_sync();
       issue_qk<D>(tS, q_u32, ring_u32 + st * C::TILE_BYTES, TILE);
       mma_commit(&mi.s_full[b]);
@@ -410,6 +414,7 @@ __device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b,
       mbar_arrive(&mi.kv_free[st]);
     }
   }
+  bool first = true;                           // no P V of this block issued yet: the first one overwrites the accumulator
   for (int j = 0; j < n; ++j) {
     const int st_v = wt.kv % NS;
     mbar_wait(&mi.kv_full[st_v], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
@@ -421,19 +426,26 @@ __device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b,
       mbar_wait(&mi.kv_full[st_k], full_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFULL);
       ++wt.kv;
     }
-    if (has_b && j < nb_b) {
-      // first half of P V as soon as keys 0..63 of P are in TMEM (no token: it is not on the
-      // other block's critical path for long, and the pipe is in order)
-      mbar_wait(&mi.p_half[b], full_par(wt.p[b]), cx.abort_flag, cx.status, W_PHALF);
-      tc_fence_after_sync();
-      issue_pv<D>(tO, tS, ring_u32 + st_v * C::TILE_BYTES, j > 0, 0, TILE / 32);
-      mbar_wait(&mi.p_full[b], full_par(wt.p[b]), cx.abort_flag, cx.status, W_PFULL);
-      ++wt.p[b];
+    const bool pv_now = takes_part(j), qk_next = takes_part(j + 1);
+    if (pv_now || qk_next) {
+      if (pv_now) {
+        // first half of P V as soon as keys 0..63 of P are in TMEM (no token: it is not on the
+        // other block's critical path for long, and the pipe is in order)
+        mbar_wait(&mi.p_half[b], full_par(wt.p[b]), cx.abort_flag, cx.status, W_PHALF);
+        tc_fence_after_sync();
+        issue_pv<D>(tO, tS, ring_u32 + st_v * C::TILE_BYTES, !first, 0, TILE / 32);
+        mbar_wait(&mi.p_full[b], full_par(wt.p[b]), cx.abort_flag, cx.status, W_PFULL);
+        ++wt.p[b];
+      }
       turn_take(cx, wt, b);
       tc_fence_after_sync();
-      issue_pv<D>(tO, tS, ring_u32 + st_v * C::TILE_BYTES, true, TILE / 32, TILE / 16);
-      if (j == nb_b - 1) mma_commit(&mi.o_full[b]);
-      if (j + 1 < nb_b) { issue_qk<D>(tS, q_u32, ring_u32 + st_k * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
+      if (pv_now) {
+        issue_pv<D>(tO, tS, ring_u32 + st_v * C::TILE_BYTES, true, TILE / 32, TILE / 16);
+        first = false;
+        if (j == last) mma_commit(&mi.o_full[b]);
+      }
+      // S of this block's next tile overwrites S / P of its previous one: the pipe runs the P V above first
+      if (qk_next) { issue_qk<D>(tS, q_u32, ring_u32 + st_k * C::TILE_BYTES, TILE); mma_commit(&mi.s_full[b]); }
       turn_pass(cx, wt, b);
       mma_commit(&mi.kv_free[st_v]);
       if (more) mma_commit(&mi.kv_free[st_k]);
@@ -447,20 +459,22 @@ __device__ __forceinline__ void mma_flash_block(const Ctx& cx, Waits& wt, int b,
   if (has_b) ++wt.acc[b];
 }
 
-// softmax group: online softmax over n key tiles for this thread's row; vis(j) = visible
-// columns of tile j.  Leaves (m_used, l_run); the accumulator O_b stays in TMEM.
+// softmax group: online softmax over the key tiles of this block (all n, or with `alternate` those of parity b)
+// for this thread's row; vis(j) = visible columns of tile j.  Leaves (m_used, l_run); the accumulator O_b stays
+// in TMEM.
 template <int D, class VisFn>
 __device__ __forceinline__ void wg_flash_loop(const Ctx& cx, uint32_t& n_s, uint32_t& n_o, int b, uint32_t tS,
                                               uint32_t tO, int n, float scale_log2, VisFn vis, float& m_used,
-                                              float& l_run) {
+                                              float& l_run, bool alternate = false) {
   Misc& mi = *cx.mi;
   m_used = -INFINITY;
   l_run = 0.0f;
-  for (int j = 0; j < n; ++j) {
+  const int j0 = alternate ? b : 0, step = alternate ? 2 : 1;
+  for (int j = j0; j < n; j += step) {
     mbar_wait(&mi.s_full[b], full_par(n_s), cx.abort_flag, cx.status, W_SFULL);
     ++n_s;
     tc_fence_after_sync();
-    softmax_tile<D>(tS, tO, vis(j), j == 0, scale_log2, m_used, l_run, &mi.p_half[b]);
+    softmax_tile<D>(tS, tO, vis(j), j == j0, scale_log2, m_used, l_run, &mi.p_half[b]);
     tc_fence_before_sync();
     warp_arrive(&mi.p_full[b]);
   }
@@ -746,7 +760,10 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 // ====================================================================================
 //                          PARALLEL (GLOBAL) ATTENTION KERNEL
 // ====================================================================================
-// Queries arrive rotated (RoPE pre-pass).  Item = (sequence, kv-head, row group, key split).  The rows of an item are the w window
+// Queries arrive rotated (RoPE pre-pass).  Item = (sequence, kv-head, row group, key split).
+// When the rows of an item fill one block only (G * w <= 128, e.g. a decoding step), both blocks hold those
+// rows and take alternate key tiles, each with its own running maximum, sum and accumulator: two softmax
+// streams per CTA instead of one, merged afterwards like two key splits.  The rows of an item are the w window
 // queries of up to 256/w q-heads of one kv-head, packed head-major into the two 128-row
 // blocks; both blocks stream the same cache tiles, and the last split appends the
 // window's own keys (causal inside the window).
@@ -794,6 +811,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
     const int rows_total = heads * prm.w;
     d.rows[0] = rows_total < TILE ? rows_total : TILE;
     d.rows[1] = rows_total > TILE ? rows_total - TILE : 0;
+    if (prm.alt) d.rows[1] = d.rows[0];           // one block of rows: both blocks hold it and share the key tiles
     d.j0 = d.split * prm.tiles_per_split;
     const int j1 = (d.j0 + prm.tiles_per_split) < prm.n_cache_tiles ? (d.j0 + prm.tiles_per_split) : prm.n_cache_tiles;
     d.n_cache = j1 - d.j0;
@@ -814,7 +832,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
           mbar_wait(&mi.q_free[b], free_par(wt.q[b]), cx.abort_flag, cx.status, W_QFREE);
           mbar_arrive_expect_tx(&mi.q_full[b], d.rows[b] * D * 2);
           for (int r0 = 0; r0 < d.rows[b]; r0 += prm.w) {
-            const int g = d.g0 + (b * TILE + r0) / prm.w;
+            const int g = d.g0 + ((prm.alt ? 0 : b * TILE) + r0) / prm.w;
             for (int a = 0; a < C::ATOMS; ++a)
               tma_load_4d(cx.sQ[b] + a * 16384 + r0 * 128, &tm_qw, &mi.q_full[b], a * 64, d.hkv * G + g, 0, d.seq);
           }
@@ -841,7 +859,7 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
         if (item == ITEM_DONE) break;
         const Dec d = decode(item);
         const bool has_b = d.rows[b] > 0;
-        mma_flash_block<D>(cx, wt, b, has_b, has_b ? d.n : 0, d.n);
+        mma_flash_block<D>(cx, wt, b, has_b, has_b ? d.n : 0, d.n, prm.alt != 0);
       }
       mma_commit(&mi.mma_done);
     }
@@ -866,12 +884,12 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
                          const int left = prm.Nk - (d.j0 + jj) * TILE;             // ragged last cache tile
                          return left < TILE ? left : TILE;
                        },
-                       m_used, l_run);
+                       m_used, l_run, prm.alt != 0);
       if (r == 0) mbar_arrive(&mi.q_free[b]);                 // all MMAs that read sQ[b] have completed
-      const int g = d.g0 + (b * TILE + r) / prm.w;
+      const int g = d.g0 + ((prm.alt ? 0 : b * TILE) + r) / prm.w;
       const int h = d.hkv * G + g;
       const bool valid = r < rows_b;
-      if (prm.n_split == 1) {
+      if (prm.n_part == 1) {
         const float inv_l = 1.0f / l_run;
         uint4* dst = reinterpret_cast<uint4*>(prm.out + (((size_t)d.seq * prm.w + wi) * prm.Hq + h) * D);
 #pragma unroll
@@ -893,7 +911,8 @@ parallel_attn_kernel(const __grid_constant__ CUtensorMap tm_qw, const __grid_con
         if (valid && prm.lse_out)
           prm.lse_out[((size_t)d.seq * prm.Hq + h) * prm.w + wi] = (m_used + log2f(l_run)) * 0.6931471805599453f;
       } else {
-        const size_t prow = (((size_t)d.seq * prm.Hq + h) * prm.n_split + d.split) * prm.w + wi;
+        const int part = prm.alt ? 2 * d.split + b : d.split;   // partial result of this block
+        const size_t prow = (((size_t)d.seq * prm.Hq + h) * prm.n_part + part) * prm.w + wi;
         uint4* dst = reinterpret_cast<uint4*>(prm.part_o + prow * D);
 #pragma unroll
         for (int q = 0; q < D / 32; ++q) {
@@ -986,11 +1005,11 @@ static cudaError_t launch_parallel_t(const CUtensorMap* maps, const ParallelPara
   parallel_attn_kernel<D><<<grid, NUM_THREADS, Cfg<D>::SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (prm.n_split > 1) {
+  if (prm.n_part > 1) {
     const int rows = prm.B * prm.Hq * prm.w;
     note_launch();
     parallel_merge_kernel<D><<<(rows + 7) / 8, 256, 0, st>>>(prm.part_o, prm.part_ml, prm.B * prm.Hq, prm.w, prm.Hq,
-                                                            prm.n_split, prm.out, prm.lse_out);
+                                                            prm.n_part, prm.out, prm.lse_out);
     e = cudaGetLastError();
   }
   return e;

@@ -30,9 +30,11 @@ struct ParallelParams {
   int B, w, Hq, Hkv, Nk;
   int Gs, n_rg;                  // q-heads per row group (Gs * w <= 256), row groups per kv-head
   int n_cache_tiles, n_split, tiles_per_split;
+  int alt;                       // 1: the item's rows fit one block; the two blocks take alternate key tiles of the split
+  int n_part;                    // partial results per (sequence, q-head): n_split, or 2 * n_split with alt
   float scale_log2;
-  float* part_o;                 // [B,Hq,n_split,w,d] fp32 unnormalised partial outputs (n_split > 1)
-  float* part_ml;                // [B,Hq,n_split,w,2] (running max in log2 units, sum)
+  float* part_o;                 // [B,Hq,n_part,w,d] fp32 unnormalised partial outputs (n_part > 1)
+  float* part_ml;                // [B,Hq,n_part,w,2] (running max in log2 units, sum)
   __nv_bfloat16* out;            // [B,w,Hq,d]
   float* lse_out;                // [B,Hq,w] or null
   int* status;
