@@ -345,8 +345,9 @@ __device__ __forceinline__ void producer_ring_tile(const Ctx& cx, Waits& wt, con
                                                    int c3) {
   using C = Cfg<D>;
   Misc& mi = *cx.mi;
+  if (*cx.abort_flag) return;                  // a wait has run out: no copy is issued into a ring that nobody drains
   const int st = wt.kv % NS;
-  mbar_wait(&mi.kv_free[st], free_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFREE);
+  if (!mbar_wait(&mi.kv_free[st], free_par(wt.kv / NS), cx.abort_flag, cx.status, W_KVFREE)) return;
   mbar_arrive_expect_tx(&mi.kv_full[st], C::TILE_BYTES);
   for (int a = 0; a < C::ATOMS; ++a)
     tma_load_4d(cx.ring + st * C::TILE_BYTES + a * 16384, tmap, &mi.kv_full[st], a * 64, c1, c2, c3);

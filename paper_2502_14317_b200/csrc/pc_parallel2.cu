@@ -155,7 +155,9 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc); tma_prefetch_desc(&tm_kw);
       tma_prefetch_desc(&tm_vw);
       uint32_t cQ = 0, cK = 0, cV = 0;
-      for (int item = pair_id; item < n_items; item += n_pairs) {
+      // Once a wait has run out (abort flag) no new work is started: every role leaves its loops at the next item,
+      // this one also at the next tile, so that no copy is issued into a ring that nobody drains any more.
+      for (int item = pair_id; item < n_items && !*cx.abort_flag; item += n_pairs) {
         const Item3 it = decode_item3(prm, item);
         {
           const int qb = cQ & 1;
@@ -168,7 +170,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                                it.seq);
           ++cQ;
         }
-        for (int j = 0; j < n_tiles; ++j) {
+        for (int j = 0; j < n_tiles && !*cx.abort_flag; ++j) {
           {
             const int s = cK % NKS;
             WAIT3(&mi.k_free[s], free_par(cK / NKS), W3_KFREE);
@@ -213,7 +215,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       const uint32_t idesc_qk = make_idesc_bf16_f32(256, TILE, false, false);
       const uint32_t rk_u32 = smem_u32(cx.rK);
       uint32_t cQ = 0, cK = 0, cS = 0;
-      for (int item = pair_id; item < n_items; item += n_pairs) {
+      for (int item = pair_id; item < n_items && !*cx.abort_flag; item += n_pairs) {
         const int qb = cQ & 1;
         WAIT3(&mi.q_full[qb], full_par(cQ >> 1), W3_QFULL);             // the query tiles of both CTAs have landed
         ++cQ;
@@ -248,7 +250,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       constexpr uint32_t idesc_pv = make_idesc_bf16_f32(256, D, false, true);
       const uint32_t rv_u32 = smem_u32(cx.rV);
       uint32_t cS = 0, n_done = 0, n_turn = 0;
-      for (int item = pair_id; item < n_items; item += n_pairs) {
+      for (int item = pair_id; item < n_items && !*cx.abort_flag; item += n_pairs) {
         WAIT3(&mi.acc_free, free_par(n_done), W3_ACCFREE);                     // accumulator of the previous item read out
         for (int j = 0; j < n_tiles; ++j, ++cS) {
           if ((int)(cS & 1) != me) continue;
@@ -299,7 +301,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         store_pending = -1;
       }
     };
-    for (int item = pair_id; item < n_items; item += n_pairs) {
+    for (int item = pair_id; item < n_items && !*cx.abort_flag; item += n_pairs) {
       const Item3 it = decode_item3(prm, item);
       const int h = it.h0 + (int)rank * prm.hpc + h_local;
       const int qb = cQ & 1;                                 // this item's query buffer (its output is staged there)

@@ -257,7 +257,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kh); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
       tma_prefetch_desc(&tm_qw);
       uint32_t cQ = 0, cK = 0, cV = 0;
-      for (int item = pair_id; item < n_items; item += n_pairs) {
+      // Once a wait has run out (abort flag) no new work is started: every role leaves its loops at the next item,
+      // this one also at the next tile, so that no copy is issued into a ring that nobody drains any more.
+      for (int item = pair_id; item < n_items && !*cx.abort_flag; item += n_pairs) {
         int group, within, c, hkv;
         sch.d_ipg.divmod(item, group, within);
         sch.d_hkv.divmod(group, c, hkv);
@@ -274,7 +276,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int a = 0; a < 2; ++a) tma_load_4d_pair(cx.sQ[qb] + a * 16384, &tm_q, bar, a * 64, bk.h, bk.t * TILE, c);
             ++cQ;
           }
-          for (int j = 0; j < bk.n; ++j) {
+          for (int j = 0; j < bk.n && !*cx.abort_flag; ++j) {
             {
               const int s = cK % NKS;
               WAIT2(&mi.k_free[s], free_par(cK / NKS), W2_KFREE);
@@ -317,7 +319,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               if (leader) mbar_arrive(&mi.k_full[s]);
               ++cK;
             }
-            for (int jj = 0; jj < n_sweep_tiles; ++jj) {
+            for (int jj = 0; jj < n_sweep_tiles && !*cx.abort_flag; ++jj) {
               const int tile = 2 * jj + (int)rank;
               for (int a = 0; a < 2; ++a) {
                 const int s = cK % NKS;
@@ -352,7 +354,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint32_t idesc_sw = make_idesc_bf16_f32(256, 2 * rows_half, false, false);
       const uint32_t rk_u32 = smem_u32(cx.rK);
       uint32_t cQ = 0, cK = 0, cS = 0, cT = 0, n_done = 0;
-      for (int item = pair_id; item < n_items; item += n_pairs) {
+      for (int item = pair_id; item < n_items && !*cx.abort_flag; item += n_pairs) {
         int group, within, c, hkv;
         sch.d_ipg.divmod(item, group, within);
         sch.d_hkv.divmod(group, c, hkv);
@@ -437,7 +439,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       constexpr uint32_t idesc_pv = make_idesc_bf16_f32(256, D, false, true);
       const uint32_t rv_u32 = smem_u32(cx.rV);
       uint32_t cS = 0, n_done = 0, n_turn = 0;
-      for (int item = pair_id; item < n_items; item += n_pairs) {
+      for (int item = pair_id; item < n_items && !*cx.abort_flag; item += n_pairs) {
         int group, within, c, hkv;
         sch.d_ipg.divmod(item, group, within);
         sch.d_hkv.divmod(group, c, hkv);
@@ -499,7 +501,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         store_pending = -1;
       }
     };
-    for (int item = pair_id; item < n_items; item += n_pairs) {
+    for (int item = pair_id; item < n_items && !*cx.abort_flag; item += n_pairs) {
       int group, within, c, hkv;
       sch.d_ipg.divmod(item, group, within);
       sch.d_hkv.divmod(group, c, hkv);
