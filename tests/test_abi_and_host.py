@@ -65,6 +65,10 @@ def test_workspace_queries_are_host_only(lib):
     # (max, sum) per split besides the tables and the rotated queries
     fixed = 256 + 64 * 64 * 16 + 2 * 64 * 32 * 16 + 1 * 64 * 32 * 128 * 2
     assert binding.parallel_attn_workspace_bytes(1, 64, 32, 8, 128, 16384) == fixed + 16 * 32 * 64 * (128 + 2) * 4
+    # a decoding step (one query token per sequence): the four rows of a kv-head fill one block only, so both blocks of
+    # a CTA take alternate key tiles and every one of the 2 key splits leaves two partial results per (sequence, q-head)
+    fixed = 256 + 1 * 64 * 16 + 2 * 1 * 32 * 16 + 64 * 1 * 32 * 128 * 2
+    assert binding.parallel_attn_workspace_bytes(64, 1, 32, 8, 128, 16384) == fixed + 4 * 64 * 32 * 1 * (128 + 2) * 4
     assert binding.parallel_attn_workspace_bytes(64, 64, 32, 8, 100, 16384) == 0
 
 
