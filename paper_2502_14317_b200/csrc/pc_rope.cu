@@ -62,22 +62,25 @@ __global__ void __launch_bounds__(256, 4) rope_rows_kernel(const uint16_t* __res
   float4 hi[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) hi[i] = __ldg(hi_row + g * 4 + i);
-  const long long step_src = (long long)h_step * s_head;
+  const int zs = gridDim.z;                                 // small inputs: the head passes are dealt out over grid.z
+  const long long step_src = (long long)h_step * zs * s_head;
+  const size_t step_dst = (size_t)h_step * zs * d;
   const int n_pass = (H + h_step - 1) / h_step;
+  const int h_mine = h_first + (int)blockIdx.z * h_step;    // this thread's head in its first pass
   for (int c = blockIdx.y; c < C; c += gridDim.y) {
-    const uint16_t* src = x + (long long)c * s_chunk + (long long)p * s_tok + (long long)h_first * s_head + g * 8;
+    const uint16_t* src = x + (long long)c * s_chunk + (long long)p * s_tok + (long long)h_mine * s_head + g * 8;
     uint16_t* const dst_tok = y + ((size_t)c * L + p) * H * d;
-    uint16_t* dst = dst_tok + (size_t)h_first * d + g * 8;
+    uint16_t* dst = dst_tok + (size_t)h_mine * d + g * 8;
     uint4 n1 = make_uint4(0, 0, 0, 0), n2 = make_uint4(0, 0, 0, 0);
-    if (h_first < H) {
+    if (h_mine < H) {
       n1 = __ldg(reinterpret_cast<const uint4*>(src));
       n2 = __ldg(reinterpret_cast<const uint4*>(src + half));
     }
 #pragma unroll 1
-    for (int ps = 0; ps < n_pass; ++ps, src += step_src, dst += (size_t)h_step * d) {
+    for (int ps = blockIdx.z; ps < n_pass; ps += zs, src += step_src, dst += step_dst) {
       const bool active = h_first + ps * h_step < H;
       const uint4 x1 = n1, x2 = n2;
-      if (h_first + (ps + 1) * h_step < H) {                // the next pass's row is in flight during this one's arithmetic
+      if (ps + zs < n_pass && h_first + (ps + zs) * h_step < H) {                // the next pass's row is in flight during this one's arithmetic
         n1 = __ldg(reinterpret_cast<const uint4*>(src + step_src));
         n2 = __ldg(reinterpret_cast<const uint4*>(src + step_src + half));
       } else {
@@ -128,7 +131,12 @@ void launch_rope_rows(const void* x, const long long x_stride[3], void* y, const
   // a slice of the chunks per block: the table entries are reused over the slice; enough blocks to fill the GPU
   int ny = (4736 + bx - 1) / bx;
   ny = ny < 1 ? 1 : (ny > C ? C : ny);
-  dim3 grid((unsigned)bx, (unsigned)ny);
+  // a few positions and chunks only (the query window of one sequence): the passes over the heads, which a warp
+  // would otherwise walk one after the other, become blocks of their own
+  const int n_pass = (H + 32 / (d / 16) - 1) / (32 / (d / 16));
+  int nz = bx * ny < 592 ? 592 / (bx * ny) : 1;
+  nz = nz > n_pass ? n_pass : (nz < 1 ? 1 : nz);
+  dim3 grid((unsigned)bx, (unsigned)ny, (unsigned)nz);
   note_launch();
   rope_rows_kernel<<<grid, 256, 0, st>>>((const uint16_t*)x, x_stride[0], x_stride[1], x_stride[2], (uint16_t*)y, tab_hi,
                                          tab_lo, tab, C, L, H, d);
