@@ -17,6 +17,9 @@
 // While group 0 runs its softmax the tensor core works for group 1 and vice versa.
 // The running maximum is only raised when it grows by more than 2^8 (lazy rescale), so
 // the accumulator is rarely touched between tiles.
+// Queries and keys arrive rotated (the RoPE pre-pass of pc_rope.cu runs before these kernels).
+// In the parallel attention an item whose rows fill one block only (a decoding step) is run by
+// BOTH groups on alternate key tiles and merged afterwards, like two key splits.
 //
 // Window scores (prefill only): the item that owns the last query tiles of a
 // (chunk, kv-head) group runs them for all G q-heads, keeps the window rows' final
