@@ -25,6 +25,9 @@ def _bits(rng, shape):
     (2, 1, 8, 2, 128, 3000, 8191, 5e5),       # decoding step: one query token over the cache (+ its own key)
     (3, 2, 4, 4, 64, 500, 4094, 1e4),         # two query tokens, MHA
     (1, 4, 32, 8, 128, 16384, 8188, 5e5),     # four query tokens over a 16K cache, Llama-3 heads
+    (2, 4, 8, 2, 128, 50, 77, 1e4),           # rows fill one block: two streams; one cache tile to one, the window tile to the other
+    (5, 1, 4, 4, 64, 128, 4095, 1e4),         # decoding, MHA, head size 64, cache of exactly one tile
+    (1, 16, 8, 2, 128, 5000, 300, 5e5),       # 64 rows per kv-head, 40 cache tiles split over the CTAs, two streams each
     # batches whose 256-row groups fill the CTA pairs (head size 128, G*w a multiple of 256): the pair kernel
     (8, 64, 32, 8, 128, 300, 8128, 5e5),      # 64 groups, ragged last cache tile
     (15, 64, 32, 8, 128, 256, 8128, 5e5),     # 120 groups: two rounds per pair, cache of whole tiles
