@@ -297,6 +297,24 @@ PC_API int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, i
                          size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------
+ * Generation over the compressed cache (paper: Sec. 3.1 "Global attention" - the compressed
+ * cache is what the following generation attends over; Table 7, per-token column).
+ * pc_parallel_attn for caches stored with room to grow, followed by the append of the new
+ * entries: k_cache, v_cache [B,Hkv,Nk_cap,d], of which the first Nk entries of every
+ * (sequence, kv-head) are valid; the w new tokens (w = 1: one decoding step) attend to them
+ * and causally to themselves exactly as in pc_parallel_attn, and afterwards, on the same
+ * stream, their rotated keys and values k_win, v_win [B,w,Hkv,d] are copied to entries
+ * Nk..Nk+w-1, so that the next step calls with Nk + w and q_pos0 + w.  Entries from Nk on are
+ * never read by the attention.  PC_ERR_INVALID_ARG if Nk + w > Nk_cap.  Workspace:
+ * pc_parallel_attn_workspace_bytes(B, w, Hq, Hkv, d, Nk).  Everything else as pc_parallel_attn.
+ */
+PC_API int32_t pc_parallel_attn_append(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk,
+                                int32_t Nk_cap, const void* q_win, int32_t q_pos0, float rope_theta,
+                                float softmax_scale, void* k_cache, void* v_cache, const void* k_win,
+                                const void* v_win, void* out, float* lse_out, int32_t* status_word,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------
  * pc_parallel_attn without a workspace argument, for callers that must not allocate.
  * The paper has no counterpart of this call: it computes exactly what pc_parallel_attn
  * computes (same kernels, same split plan, same results) and exists for the callers

@@ -85,6 +85,9 @@ def load_library():
     lib.pc_parallel_attn.restype = c_int32
     lib.pc_parallel_attn.argtypes = [c_int32] * 6 + [c_void_p, c_int32, c_float, c_float] + [c_void_p] * 8 + \
                                     [c_size_t, c_void_p]
+    lib.pc_parallel_attn_append.restype = c_int32
+    lib.pc_parallel_attn_append.argtypes = [c_int32] * 7 + [c_void_p, c_int32, c_float, c_float] + [c_void_p] * 8 + \
+                                           [c_size_t, c_void_p]
     lib.pc_parallel_attn_static_scratch_bytes.restype = c_size_t
     lib.pc_parallel_attn_static_scratch_bytes.argtypes = []
     lib.pc_parallel_attn_static.restype = c_int32
@@ -381,6 +384,33 @@ def parallel_attn(q_win, k_cache, v_cache, k_win, v_win, *, q_pos0, rope_theta, 
                               _ptr(k_cache), _ptr(v_cache), _ptr(k_win), _ptr(v_win), _ptr(out), _ptr(lse_out),
                               _ptr(status), _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "pc_parallel_attn")
+    return {"out": out, "lse": lse_out, "status": status, "workspace": workspace}
+
+
+def parallel_attn_append(q_win, k_cache, v_cache, n_valid, k_win, v_win, *, q_pos0, rope_theta, softmax_scale=0.0,
+                         out=None, lse_out=None, want_lse=False, status=None, workspace=None):
+    """pc_parallel_attn_append: as parallel_attn over the first ``n_valid`` entries of k_cache / v_cache
+    [B,Hkv,Nk_cap,d]; afterwards k_win, v_win are written to entries n_valid .. n_valid + w - 1 of the caches."""
+    lib = load_library()
+    _need_cuda(q_win, k_cache, v_cache, k_win, v_win)
+    B, w, Hq, d = q_win.shape
+    Hkv, cap = k_cache.shape[1], k_cache.shape[2]
+    dev = q_win.device
+    for t in (q_win, k_cache, v_cache, k_win, v_win):
+        if not t.is_contiguous():
+            raise PcError("pc_parallel_attn_append takes contiguous tensors")
+    out = torch.empty((B, w, Hq, d), dtype=torch.bfloat16, device=dev) if out is None else out
+    if lse_out is None and want_lse:
+        lse_out = torch.empty((B, Hq, w), dtype=torch.float32, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    need = parallel_attn_workspace_bytes(B, w, Hq, Hkv, d, int(n_valid))
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    rc = lib.pc_parallel_attn_append(B, w, Hq, Hkv, d, int(n_valid), cap, _ptr(q_win), int(q_pos0), float(rope_theta),
+                                     float(softmax_scale), _ptr(k_cache), _ptr(v_cache), _ptr(k_win), _ptr(v_win),
+                                     _ptr(out), _ptr(lse_out), _ptr(status), _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "pc_parallel_attn_append")
     return {"out": out, "lse": lse_out, "status": status, "workspace": workspace}
 
 

@@ -456,12 +456,18 @@ size_t pc_parallel_attn_workspace_bytes(int32_t B, int32_t w, int32_t Hq, int32_
   return parallel_plan(B, w, Hq, Hkv, d, Nk, plan_sm_count()).total;
 }
 
-int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk, const void* q_win,
-                         int32_t q_pos0, float rope_theta, float softmax_scale, const void* k_cache,
-                         const void* v_cache, const void* k_win, const void* v_win, void* out, float* lse_out,
-                         int32_t* status_word, void* workspace, size_t workspace_bytes, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// pc_parallel_attn over caches whose (sequence, kv-head) rows are Nk_cap entries apart (Nk of them valid)
+int32_t parallel_attn_impl(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk, int64_t Nk_cap,
+                           const void* q_win, int32_t q_pos0, float rope_theta, float softmax_scale, const void* k_cache,
+                           const void* v_cache, const void* k_win, const void* v_win, void* out, float* lse_out,
+                           int32_t* status_word, void* workspace, size_t workspace_bytes, void* stream) {
   int32_t rc = check_parallel_args(B, w, Hq, Hkv, d, Nk);
   if (rc != PC_OK) return rc;
+  if (Nk_cap < Nk || Nk_cap > (1ll << 28)) return PC_ERR_INVALID_ARG;
   if (!q_win || !k_cache || !v_cache || !k_win || !v_win || !out) return PC_ERR_INVALID_ARG;
   if (!aligned16(q_win) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_win) || !aligned16(v_win) ||
       !aligned16(out) || !aligned16(workspace))
@@ -481,7 +487,7 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   const uint64_t qw_dims[4] = {ud, (uint64_t)Hq, (uint64_t)w, (uint64_t)B};
   const uint64_t qw_str[3] = {ud, (uint64_t)Hq * ud, (uint64_t)w * Hq * ud};
   const uint64_t kc_dims[4] = {ud, (uint64_t)Nk, (uint64_t)Hkv, (uint64_t)B};
-  const uint64_t kc_str[3] = {ud, (uint64_t)Nk * ud, (uint64_t)Hkv * Nk * ud};
+  const uint64_t kc_str[3] = {ud, (uint64_t)Nk_cap * ud, (uint64_t)Hkv * (uint64_t)Nk_cap * ud};
   const uint64_t kw_dims[4] = {ud, (uint64_t)Hkv, (uint64_t)w, (uint64_t)B};
   const uint64_t kw_str[3] = {ud, (uint64_t)Hkv * ud, (uint64_t)w * Hkv * ud};
   const uint32_t box_qw[4] = {64, 1, (uint32_t)w, 1};
@@ -546,6 +552,35 @@ int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t 
   const long long n_items = (long long)B * Hkv * plan.n_rg * plan.n_split;
   const int grid = (int)(n_items < dev.sm_count ? n_items : dev.sm_count);
   if (pc::launch_parallel_attn(maps, prm, d, grid, st) != cudaSuccess) return PC_ERR_CUDA;
+  return PC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t pc_parallel_attn(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk, const void* q_win,
+                         int32_t q_pos0, float rope_theta, float softmax_scale, const void* k_cache,
+                         const void* v_cache, const void* k_win, const void* v_win, void* out, float* lse_out,
+                         int32_t* status_word, void* workspace, size_t workspace_bytes, void* stream) {
+  return parallel_attn_impl(B, w, Hq, Hkv, d, Nk, Nk, q_win, q_pos0, rope_theta, softmax_scale, k_cache, v_cache, k_win,
+                            v_win, out, lse_out, status_word, workspace, workspace_bytes, stream);
+}
+
+int32_t pc_parallel_attn_append(int32_t B, int32_t w, int32_t Hq, int32_t Hkv, int32_t d, int32_t Nk, int32_t Nk_cap,
+                                const void* q_win, int32_t q_pos0, float rope_theta, float softmax_scale, void* k_cache,
+                                void* v_cache, const void* k_win, const void* v_win, void* out, float* lse_out,
+                                int32_t* status_word, void* workspace, size_t workspace_bytes, void* stream) {
+  if (Nk_cap < 1 || (int64_t)Nk + w > (int64_t)Nk_cap) return PC_ERR_INVALID_ARG;
+  const int32_t rc = parallel_attn_impl(B, w, Hq, Hkv, d, Nk, Nk_cap, q_win, q_pos0, rope_theta, softmax_scale, k_cache,
+                                        v_cache, k_win, v_win, out, lse_out, status_word, workspace, workspace_bytes,
+                                        stream);
+  if (rc != PC_OK) return rc;
+  // the attention above reads entries below Nk only (rows behind them read as zeros and are masked): the new rows
+  // can follow on the same stream
+  if (pc::launch_append_kv(k_win, v_win, B, w, Hkv, d, Nk, Nk_cap, k_cache, v_cache, static_cast<cudaStream_t>(stream)) !=
+      cudaSuccess)
+    return PC_ERR_CUDA;
   return PC_OK;
 }
 

@@ -46,6 +46,10 @@ cudaError_t launch_gather_kv(const void* k_src, const void* v_src, const long lo
                              const int* idx, int m, int Hkv, int k, int d, void* k_out, void* v_out, int* pos_out,
                              int sm_count, bool by_slot, cudaStream_t st);
 
+// caches stored with room to grow: cache[b, hkv, Nk + i, :] = win[b, i, hkv, :] for the w new rows of every sequence
+cudaError_t launch_append_kv(const void* k_win, const void* v_win, int B, int w, int Hkv, int d, long long Nk,
+                             long long Nk_cap, void* k_cache, void* v_cache, cudaStream_t st);
+
 // ---- pc_queue.cu (online chunk queue)
 void launch_queue_init(float* q_score, int* q_chunk, int m, cudaStream_t st);
 void launch_queue_update(const float* score, int Cb, int chunk_id0, int lower_is_better, int m, float* q_score,

@@ -502,4 +502,33 @@ cudaError_t launch_gather_kv(const void* k_src, const void* v_src, const long lo
   return cudaGetLastError();
 }
 
+// Append the w new (key, value) rows of every sequence behind the Nk valid entries of caches stored with
+// room to grow: cache[b, hkv, Nk + i, :] = win[b, i, hkv, :].  One 16-byte piece per thread.
+__global__ void append_kv_kernel(const uint4* __restrict__ k_win, const uint4* __restrict__ v_win, int B, int w, int Hkv,
+                                 int lpr, long long Nk, long long Nk_cap, uint4* __restrict__ k_cache,
+                                 uint4* __restrict__ v_cache) {
+  const long long n = (long long)B * w * Hkv * lpr;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int piece = (int)(i % lpr);
+    long long x = i / lpr;
+    const int hkv = (int)(x % Hkv); x /= Hkv;
+    const int t = (int)(x % w);
+    const long long b = x / w;
+    const long long dst = ((b * Hkv + hkv) * Nk_cap + Nk + t) * lpr + piece;
+    k_cache[dst] = __ldg(k_win + i);
+    v_cache[dst] = __ldg(v_win + i);
+  }
+}
+
+cudaError_t launch_append_kv(const void* k_win, const void* v_win, int B, int w, int Hkv, int d, long long Nk,
+                             long long Nk_cap, void* k_cache, void* v_cache, cudaStream_t st) {
+  const int lpr = d / 8;
+  const long long n = (long long)B * w * Hkv * lpr;
+  const int blocks = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
+  note_launch();
+  append_kv_kernel<<<blocks < 1 ? 1 : blocks, 256, 0, st>>>((const uint4*)k_win, (const uint4*)v_win, B, w, Hkv, lpr, Nk, Nk_cap,
+                                                        (uint4*)k_cache, (uint4*)v_cache);
+  return cudaGetLastError();
+}
+
 }  // namespace pc

@@ -51,6 +51,40 @@ def test_parallel_attn_shapes(B, w, Hq, Hkv, d, Nk, q_pos0, theta):
     assert np.abs(res["lse"].cpu().numpy() - LSE).max() <= 2e-3
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,d,Nk0,cap,steps", [
+    (2, 8, 2, 128, 250, 260, (1, 1, 4, 1)),   # crosses a tile boundary of the cache (256) while generating
+    (3, 4, 4, 64, 40, 48, (1, 2, 1)),         # MHA, head size 64
+])
+def test_generation_steps_append_to_the_cache(B, Hq, Hkv, d, Nk0, cap, steps):
+    """pc_parallel_attn_append in a loop: every step attends over the entries valid so far (oracle on the same prefix)
+    and leaves its new keys / values behind them; entries further back stay as they were."""
+    import paper_2502_14317_b200 as pc
+    rng = np.random.default_rng(cap)
+    kc, vc = _bits(rng, (B, Hkv, cap, d)), _bits(rng, (B, Hkv, cap, d))    # entries >= Nk0: junk that must never be read
+    k_dev, v_dev = to_dev(kc), to_dev(vc)
+    n, pos, theta = Nk0, 1000, 1e4
+    for w in steps:
+        qw = _bits(rng, (B, w, Hq, d))
+        kw, vw = _bits(rng, (B, w, Hkv, d)), _bits(rng, (B, w, Hkv, d))
+        res = pc.parallel_attn_append(to_dev(qw), k_dev, v_dev, n, to_dev(kw), to_dev(vw), q_pos0=pos, rope_theta=theta,
+                                      want_lse=True)
+        torch.cuda.synchronize()
+        assert int(res["status"].item()) == 0
+        Fg, LSE = orc.parallel_attention(qw, pos, theta, None, np.ascontiguousarray(kc[:, :, :n]),
+                                         np.ascontiguousarray(vc[:, :, :n]), kw, vw)
+        check_attention_output(to_f64(res["out"]), Fg, f"Fg over {n} entries, {w} new")
+        assert np.abs(res["lse"].cpu().numpy() - LSE).max() <= 2e-3
+        kc[:, :, n:n + w] = kw.transpose(0, 2, 1, 3)
+        vc[:, :, n:n + w] = vw.transpose(0, 2, 1, 3)
+        assert np.array_equal(to_bits(k_dev), kc) and np.array_equal(to_bits(v_dev), vc), "cache after the append"
+        n += w
+        pos += w
+    # a step that does not fit is refused before anything is launched
+    lib = pc.load_library()
+    assert lib.pc_parallel_attn_append(B, 1, Hq, Hkv, d, cap, cap, None, 0, 1e4, 0.0, None, None, None, None, None, None,
+                                       None, None, 0, None) == -1
+
+
 def test_cfg4_slice():
     """The batch-of-compressed-caches workload at a size the oracle finishes in seconds: 2 of the 64
     sequences, full Nk = 16384 (128 key tiles), same generator."""
