@@ -554,6 +554,23 @@ def _extra_parallel(pc, torch, dev, peaks, g, out, B=64):
                              workspace=buf1.get("workspace"))
         buf1.update(r)
     us = _time_us(torch, run_dec, reps=10)
+    # ---- the same step as a generation loop runs it: caches stored with spare room, the step's key / value appended
+    cap = Nk + 64
+    kcap = torch.empty((B, Hkv, cap, d), device=dev, dtype=torch.bfloat16)
+    vcap = torch.empty((B, Hkv, cap, d), device=dev, dtype=torch.bfloat16)
+    kcap[:, :, :Nk].copy_(kc)
+    vcap[:, :, :Nk].copy_(vc)
+    buf2 = {}
+
+    def run_gen():
+        r = pc.parallel_attn_append(q1, kcap, vcap, Nk, k1, v1, q_pos0=8191, rope_theta=5e5, out=buf2.get("out"),
+                                    status=buf2.get("status"), workspace=buf2.get("workspace"))
+        buf2.update(r)
+    us_gen = _time_us(torch, run_gen, reps=10)
+    del kcap, vcap
+    out["decode_step_with_append"] = {"us": us_gen, "kv_gbs": kv_bytes / us_gen / 1e3,
+                                      "frac_of_measured_hbm": kv_bytes / us_gen / 1e3 / peaks["hbm_gbs"],
+                                      "note": "pc_parallel_attn_append, w = 1, B = %d, %d valid of %d entries" % (B, Nk, cap)}
     out["decode_step_cfg4_caches"] = {"us": us, "kv_gbs": kv_bytes / us / 1e3,
                                       "frac_of_measured_hbm": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
                                       "kv_bytes": kv_bytes, "note": "pc_parallel_attn with w = 1, B = %d, Nk = %d" % (B, Nk)}
