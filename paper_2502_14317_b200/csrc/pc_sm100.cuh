@@ -4,10 +4,10 @@
 //
 // Every wait here is bounded: after the wait limit (about a second by default) without
 // completion the waiter raises a CTA-wide abort flag and stores a code that names the
-// wait in the caller's status word; all later waits return at once, control flow (which
-// never depends on data) runs to its normal end, copies and tensor-core work in flight
-// are drained, and the kernel returns.  A bug in a barrier phase therefore cannot leave
-// the GPU spinning.
+// wait in the caller's status word; all later waits return at once, no role starts new
+// work (the loops over work items and, in the producers, over tiles test the flag), copies
+// and tensor-core work in flight are drained, and the kernel returns.  A bug in a barrier
+// phase therefore cannot leave the GPU spinning.
 #pragma once
 #include <cstdint>
 #include <cuda_bf16.h>
