@@ -188,3 +188,18 @@ def test_boundary_has_the_argument_lists_of_the_scope_table():
     assert _params("pc_parallel_attn") == ["B", "w", "Hq", "Hkv", "d", "Nk", "q_win", "q_pos0", "rope_theta",
                                            "softmax_scale", "k_cache", "v_cache", "k_win", "v_win", "out", "lse_out",
                                            "status_word", "workspace", "workspace_bytes", "stream"]
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/pc.h is the boundary for C callers: it must compile as C99 on its own, without warnings."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler here")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "use_pc.c"
+    src.write_text('#include "pc.h"\nint main(void) { return (int)sizeof(pc_prefill_desc) == 0; }\n')
+    r = subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
+                        "-I", os.path.join(root, "include"), str(src)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
