@@ -74,7 +74,9 @@ struct Ctx3 {
   int* status;
 };
 
-#define WAIT3(bar, par, code) mbar_wait((bar), (par), cx.abort_flag, cx.status, (code))
+// waits of the single-thread service roles (long pause between polls) / of the softmax warps
+#define WAIT3(bar, par, code) mbar_wait_ns<SERVICE_BACKOFF_NS>((bar), (par), cx.abort_flag, cx.status, (code))
+#define WAIT3S(bar, par, code) mbar_wait((bar), (par), cx.abort_flag, cx.status, (code))
 
 __device__ __forceinline__ void init_barriers3(Misc3& mi, int wait_kcycles) {
   for (int b = 0; b < 2; ++b) { mbar_init(&mi.q_full[b], 1); mbar_init(&mi.q_free[b], 1); }
@@ -312,7 +314,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const int owner = cS & 1;
         if (owner != hlf) continue;
         const int sb = cS % NSB;
-        WAIT3(&mi.s_full[owner][sb], full_par(cS / NSB), W3_SFULL);
+        WAIT3S(&mi.s_full[owner][sb], full_par(cS / NSB), W3_SFULL);
         tc_fence_after_sync();
         const uint32_t tS = cx.tmem + sb * TILE + lane_sel;
         uint32_t s[4][32];
@@ -342,7 +344,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const float m_tile = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3])) * scale_log2;
         float m_prev = -INFINITY;
         if (j > 0) {                                           // the partner's publication of tile j-1
-          WAIT3(&mi.m_pub[hlf ^ 1][warp & 3], full_par(n_pub_other), W3_MPUB);
+          WAIT3S(&mi.m_pub[hlf ^ 1][warp & 3], full_par(n_pub_other), W3_MPUB);
           ++n_pub_other;
           m_prev = mi.mref[(j - 1) & 1][r];
         }
@@ -362,7 +364,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           // P V of tile j cannot start before this thread publishes P.
           const float alpha = (m_prev == -INFINITY) ? 0.0f : fast_exp2(m_prev - m_new);
           const uint32_t prev = cS - 1;
-          WAIT3(&mi.v_free[prev % NVS], full_par(prev / NVS), W3_PVDONE);   // committed after P V of tile `prev`
+          WAIT3S(&mi.v_free[prev % NVS], full_par(prev / NVS), W3_PVDONE);   // committed after P V of tile `prev`
           tc_fence_after_sync();
           const uint32_t tO = cx.tmem + TM_O + lane_sel;
 #pragma unroll 1
@@ -379,7 +381,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           // the P buffer of this warpgroup is free once P V of its previous tile has run; this wait also keeps
           // the softmax at most one own tile ahead of the P V issuer, whose barriers have one phase bit
           const uint32_t prev2 = cS - 2;
-          WAIT3(&mi.v_free[prev2 % NVS], full_par(prev2 / NVS), W3_PVDONE);
+          WAIT3S(&mi.v_free[prev2 % NVS], full_par(prev2 / NVS), W3_PVDONE);
           tc_fence_after_sync();
         }
         const float neg_m = (m_new == -INFINITY) ? 0.0f : -m_new;
@@ -421,7 +423,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       {
         const int last_owner = (cS - 1) & 1;
         if (hlf != last_owner) {
-          WAIT3(&mi.m_pub[hlf ^ 1][warp & 3], full_par(n_pub_other), W3_MPUB);
+          WAIT3S(&mi.m_pub[hlf ^ 1][warp & 3], full_par(n_pub_other), W3_MPUB);
           ++n_pub_other;
         }
         const float m_fin = mi.mref[(n_tiles - 1) & 1][r];
@@ -433,7 +435,7 @@ parallel_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       finish_store();
       // ---- epilogue: combine the two partial row sums, normalise, stage bf16 rows in this item's (now idle)
       // Q buffer, TMA store (one box per head: its w window rows)
-      WAIT3(&mi.o_full, full_par(n_done), W3_OFULL);
+      WAIT3S(&mi.o_full, full_par(n_done), W3_OFULL);
       ++n_done;
       tc_fence_after_sync();
       mi.xl[hlf][r] = l_run;

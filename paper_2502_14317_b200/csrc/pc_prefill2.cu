@@ -169,7 +169,9 @@ struct Ctx2 {
   int* status;
 };
 
-#define WAIT2(bar, par, code) mbar_wait((bar), (par), cx.abort_flag, cx.status, (code))
+// waits of the single-thread service roles (long pause between polls) / of the softmax warps
+#define WAIT2(bar, par, code) mbar_wait_ns<SERVICE_BACKOFF_NS>((bar), (par), cx.abort_flag, cx.status, (code))
+#define WAIT2S(bar, par, code) mbar_wait((bar), (par), cx.abort_flag, cx.status, (code))
 
 // wait whose completion also makes the peer CTA's earlier shared-memory writes visible
 __device__ __forceinline__ void mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
@@ -523,7 +525,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int owner = cS & 1;
           if (owner != hlf) continue;
           const int sb = cS % NSB;
-          WAIT2(&mi.s_full[owner][sb], full_par(cS / NSB), W2_SFULL);
+          WAIT2S(&mi.s_full[owner][sb], full_par(cS / NSB), W2_SFULL);
           tc_fence_after_sync();
           const uint32_t tS = cx.tmem + sb * TILE + lane_sel;
           uint32_t s[4][32];
@@ -553,7 +555,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           // reference maximum after tile j-1 (published by the other warpgroup)
           float m_prev = -INFINITY;
           if (j > 0) {                                         // the partner's publication of tile j-1
-            WAIT2(&mi.m_pub[hlf ^ 1][warp & 3], full_par(n_pub_other), W2_MPUB);
+            WAIT2S(&mi.m_pub[hlf ^ 1][warp & 3], full_par(n_pub_other), W2_MPUB);
             ++n_pub_other;
             m_prev = mi.mref[(j - 1) & 1][r];
           }
@@ -574,7 +576,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // this thread publishes P.
             const float alpha = (m_prev == -INFINITY) ? 0.0f : fast_exp2(m_prev - m_new);
             const uint32_t prev = cS - 1;
-            WAIT2(&mi.v_free[prev % NVS], full_par(prev / NVS), W2_PVDONE);   // committed after P V of tile `prev`
+            WAIT2S(&mi.v_free[prev % NVS], full_par(prev / NVS), W2_PVDONE);   // committed after P V of tile `prev`
             tc_fence_after_sync();
             const uint32_t tO = cx.tmem + TM_O + lane_sel;
 #pragma unroll 1
@@ -591,7 +593,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // the P buffer of this warpgroup is free once P V of its previous tile has run; this wait also keeps
             // the softmax at most one own tile ahead of the P V issuer, whose barriers have one phase bit
             const uint32_t prev2 = cS - 2;
-            WAIT2(&mi.v_free[prev2 % NVS], full_par(prev2 / NVS), W2_PVDONE);
+            WAIT2S(&mi.v_free[prev2 % NVS], full_par(prev2 / NVS), W2_PVDONE);
             tc_fence_after_sync();
           }
           const float neg_m = (m_new == -INFINITY) ? 0.0f : -m_new;
@@ -633,7 +635,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         {
           const int last_owner = (cS - 1) & 1;
           if (hlf != last_owner) {
-            WAIT2(&mi.m_pub[hlf ^ 1][warp & 3], full_par(n_pub_other), W2_MPUB);
+            WAIT2S(&mi.m_pub[hlf ^ 1][warp & 3], full_par(n_pub_other), W2_MPUB);
             ++n_pub_other;
           }
           const float m_fin = mi.mref[(bk.n - 1) & 1][r];
@@ -646,7 +648,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         finish_store();
         // ---- epilogue: combine the two half-row sums, normalise, stage bf16 rows in this block's
         // (now idle) Q buffer, TMA store
-        WAIT2(&mi.o_full, full_par(n_done), W2_OFULL);
+        WAIT2S(&mi.o_full, full_par(n_done), W2_OFULL);
         ++n_done;
         tc_fence_after_sync();
         mi.xl[hlf][r] = l_run;
@@ -715,7 +717,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int g_base = u * 2 * sch.hp + hlf * sch.hp;
           for (int jj = 0; jj < n_sweep_tiles; ++jj) {
             const int e = cT & 1;
-            WAIT2(&mi.t_full[e], full_par(cT >> 1), W2_TFULL);
+            WAIT2S(&mi.t_full[e], full_par(cT >> 1), W2_TFULL);
             tc_fence_after_sync();
             const int key = (2 * jj + (int)rank) * TILE + r;
             const bool need_mask = (2 * jj + (int)rank) * TILE + TILE - 1 > w0;

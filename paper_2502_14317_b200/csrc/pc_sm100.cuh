@@ -17,6 +17,11 @@ namespace pc {
 
 constexpr int WAIT_LIMIT_KCYCLES = 1 << 21;              // default wait limit in units of 1024 cycles: ~1 s at B200 clocks
 constexpr unsigned SPIN_BACKOFF_NS = 20;                 // pause between two polls of a barrier
+// The single-thread roles of the CTA-pair kernels (producer, issuers) wait much longer per poll: their waits last
+// thousands of cycles, a wake-up a few hundred cycles late costs them nothing, and every poll they do not make
+// leaves an issue slot to the softmax warp that shares their scheduler (measured: 1.2 % on the 128K shape; 640 ns
+// is too long, and for the softmax warps themselves 0, 20 or 80 ns make no difference).
+constexpr unsigned SERVICE_BACKOFF_NS = 320;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -52,14 +57,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // flag and the wait limit in units of 1024 cycles.  Once the flag is non-zero every wait
 // returns immediately (the result data is then garbage and the status word says so).
 // Returns false if the wait gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status_word, int where) {
+// NS: pause between two polls.
+template <unsigned NS>
+__device__ __forceinline__ bool mbar_wait_ns(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                             int* status_word, int where) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (SPIN_BACKOFF_NS > 0) __nanosleep(SPIN_BACKOFF_NS);   // a hot spin takes issue slots from the warps that share the scheduler
+    if (NS > 0) __nanosleep(NS);                             // a hot spin takes issue slots from the warps that share the scheduler
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > (static_cast<long long>(abort_flag[1]) << 10)) {
@@ -69,6 +76,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
+}
+
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status_word, int where) {
+  return mbar_wait_ns<SPIN_BACKOFF_NS>(bar, parity, abort_flag, status_word, where);
 }
 
 // Wait that ignores the abort flag (used only to drain copies and tensor-core work in flight before
