@@ -127,3 +127,35 @@ def test_cfg4_batch_of_compressed_caches():
                                          inp["v_cache"][s], inp["k_win"][s], inp["v_win"][s])
         check_attention_output(out[s], Fg, f"Fg seq {b}")
         assert np.abs(lse[s] - LSE).max() <= 2e-3
+
+
+def test_cfg4_decoding_step_over_the_full_batch():
+    """One generation step over the same 64 compressed caches (one query token per sequence, 4.3 GB of K/V): the
+    launch configuration the bench times (two key splits, two softmax streams per CTA, merge), every sequence
+    against the oracle; then the same step through pc_parallel_attn_append on caches with spare room."""
+    import paper_2502_14317_b200 as pc
+    cfg = pc_inputs.get_config("cfg4")
+    inp = pc_inputs.make_parallel_attn_inputs(cfg)
+    q1 = np.ascontiguousarray(inp["q_win"][:, :1])
+    k1, v1 = np.ascontiguousarray(inp["k_win"][:, :1]), np.ascontiguousarray(inp["v_win"][:, :1])
+    kc, vc = to_dev(inp["k_cache"]), to_dev(inp["v_cache"])
+    res = pc.parallel_attn(to_dev(q1), kc, vc, to_dev(k1), to_dev(v1), q_pos0=cfg.q_pos0, rope_theta=cfg.rope_theta,
+                           want_lse=True)
+    torch.cuda.synchronize()
+    assert int(res["status"].item()) == 0
+    Fg, LSE = orc.parallel_attention(q1, cfg.q_pos0, cfg.rope_theta, None, inp["k_cache"], inp["v_cache"], k1, v1)
+    check_attention_output(to_f64(res["out"]), Fg, "Fg, decoding step, 64 sequences")
+    assert np.abs(res["lse"].cpu().numpy() - LSE).max() <= 2e-3
+    B, Hkv, Nk, d = inp["k_cache"].shape
+    cap = Nk + 8
+    kcap = torch.zeros((B, Hkv, cap, d), dtype=torch.bfloat16, device="cuda")
+    vcap = torch.zeros((B, Hkv, cap, d), dtype=torch.bfloat16, device="cuda")
+    kcap[:, :, :Nk].copy_(kc)
+    vcap[:, :, :Nk].copy_(vc)
+    res2 = pc.parallel_attn_append(to_dev(q1), kcap, vcap, Nk, to_dev(k1), to_dev(v1), q_pos0=cfg.q_pos0,
+                                   rope_theta=cfg.rope_theta)
+    torch.cuda.synchronize()
+    assert int(res2["status"].item()) == 0
+    assert torch.equal(res2["out"], res["out"]), "same step, caches with spare room"
+    assert np.array_equal(to_bits(kcap[:, :, Nk]), k1[:, 0]) and np.array_equal(to_bits(vcap[:, :, Nk]), v1[:, 0])
+    assert int(kcap[:, :, Nk + 1:].abs().max().item()) == 0
