@@ -518,7 +518,23 @@ def extra_measurements(pc, torch, dev, peaks, only=None, select_chunks=8192, par
         _extra_select(pc, torch, dev, peaks, g, out, select_chunks)
     if only in (None, "gather"):
         _extra_gather(pc, torch, dev, peaks, g, out)
+    if only in (None, "rope"):
+        _extra_rope(pc, torch, dev, peaks, g, out)
     return out
+
+
+def _extra_rope(pc, torch, dev, peaks, g, out):
+    # ---- the RoPE pre-pass alone (pc_rope_position_reuse: table kernel + rotation pass), query and key tensors of cfg1
+    for name, shape in (("rope_queries_cfg1", (16, 8192, 32, 128)), ("rope_keys_cfg1", (16, 8192, 8, 128))):
+        x = torch.randn(shape, device=dev, generator=g).bfloat16()
+        y = torch.empty_like(x)
+        lib = pc.load_library()
+        ws = torch.empty(int(lib.pc_rope_position_reuse_workspace_bytes(shape[1], shape[3])), dtype=torch.uint8, device=dev)
+        us = _time_us(torch, lambda: pc.rope_position_reuse(x, rope_theta=5e5, out=y, workspace=ws), reps=10)
+        nbytes = 2.0 * x.numel() * 2
+        out[name] = {"us": us, "algorithmic_bytes": nbytes, "gbs": nbytes / us / 1e3,
+                     "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+        del x, y, ws
 
 
 def _extra_parallel(pc, torch, dev, peaks, g, out, B=64):
@@ -618,7 +634,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the single-call timings of cfg4 / scaled select / cfg2 gather")
     ap.add_argument("--parallel-batch", type=int, default=64,
                     help="sequences of the parallel-attention measurement (smaller for an ncu capture)")
-    ap.add_argument("--extra-only", default=None, choices=["parallel", "select", "gather", "prefill"],
+    ap.add_argument("--extra-only", default=None, choices=["parallel", "select", "gather", "prefill", "rope"],
                     help="run only that single-call measurement and print it (no step loop; e.g. for an ncu capture)")
     ap.add_argument("--select-chunks", type=int, default=8192,
                     help="rows / 8 of the scaled token top-k measurement (smaller for an ncu capture)")
